@@ -1,0 +1,263 @@
+#!/usr/bin/env python
+"""Benchmark: adjoint-gradient tokens/s per SSM layer at T=65,536, Tbar=2,048 (workload C3).
+
+One "step" = one as_adjoint_grad call (projections, segment pre-pass, carries, main adjoint kernel,
+weight-gradient and input-gradient contractions) on one synthetic batch.  Prints ONE JSON line.
+`--impl reference` times the fp64 CPU oracle (a deliberately plain program) on a bounded sample.
+With --gpus N > 1 (under torchrun) every rank runs an independent replica: the path has no
+cross-GPU exchange.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "adjoint-gradient tokens/sec per SSM layer (T=64K, Tbar=2K)"
+UNIT = "tokens/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks / throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+                for n, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except (ValueError, IndexError):
+                continue
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample_tokens_per_s(w, sample_T, verbose=False):
+    """Time the fp64 oracle (as it stands) on a bounded sample: batch element 0, first sample_T tokens."""
+    import numpy as np
+    import torch
+    from oracle import ssm_oracle as O
+    from paper_2501_00692_b200 import synth
+    ws = synth.custom_workload(w.name + "-sample", w.config, 1, sample_T, w.d_model, w.d_state, 1,
+                               min(w.tbar, sample_T), w.io)
+    theta = {k: synth.to_f64(v) for k, v in synth.layer_params(ws, 0, "cpu").items()}
+    x, dy = synth.activations(ws, "cpu")
+    x, dy = synth.to_f64(x), synth.to_f64(dy)
+    t0 = time.perf_counter()
+    O.batched(O.adjoint_grad, theta, x, dy, ws.tbar, tier="block")
+    dt = time.perf_counter() - t0
+    return sample_T / dt, dt, torch.get_num_threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2501_00692_b200 import synth
+    w = synth.WORKLOADS[args.workload]
+    sample_T = args.cpu_sample_tokens
+    vals = []
+    for i in range(args.warmup + args.steps):
+        tps, dt, threads = oracle_sample_tokens_per_s(w, sample_T)
+        if i >= args.warmup:
+            vals.append((tps, dt))
+    tps = sum(v[0] for v in vals) / len(vals)
+    ms = 1e3 * sum(v[1] for v in vals) / len(vals)
+    sample = f"batch element 0, first {sample_T} tokens of {w.name}, Tbar=min({w.tbar},{sample_T}), all {w.d_model} channels"
+    line = {"impl": "reference", "metric": METRIC, "value": tps, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "batch": 1, "seq_len": sample_T, "d_model": w.d_model,
+                       "d_state": w.d_state, "tbar": min(w.tbar, sample_T)},
+            "cpu_baseline": {"value": tps, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": tps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C3")
+    ap.add_argument("--cpu-sample-tokens", type=int, default=16384)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+    if args.impl == "reference":
+        args.warmup = min(args.warmup, 1); args.steps = min(args.steps, 3)
+        return run_reference(args)
+    args.warmup = max(args.warmup, 3)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2501_00692_b200 import binding as B
+    from paper_2501_00692_b200 import synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    B.lib()   # raises if the CUDA library is missing: there is no fallback
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    w = synth.WORKLOADS[args.workload]
+    theta = synth.layer_params(w, 0, dev)
+    x, dy = synth.activations(w, dev)
+    sh = B.shape_of(x, w.d_state)
+    _, gbytes = B.as_workspace_bytes(sh, w.tbar)
+    ws = B.alloc_workspace(gbytes, dev)
+    grads = B.alloc_grads(sh, dev)
+    tokens = w.batch * w.seqlen
+
+    def step():
+        B.as_adjoint_grad(sh, theta, x, dy, w.tbar, grads, ws)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    assert B.as_check_status(ws) == 0
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    # ---- device-resident timing --------------------------------------------------------------
+    B.as_launch_count(reset=True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier(); torch.cuda.synchronize()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize(); barrier()
+    launches = B.as_launch_count()
+    ms = e0.elapsed_time(e1) / args.steps
+    # ---- per-phase timing (library-side CUDA events on the launching stream) ---------------------
+    B.as_set_timing(True)
+    phase = {k: 0.0 for k in B.PHASES}
+    for _ in range(args.steps):
+        step()
+        for k, v in B.as_get_timing().items():
+            phase[k] += v / args.steps
+    B.as_set_timing(False)
+    clocks = sampler.stop() if rank == 0 else None
+    # ---- end to end: pinned host inputs -> device, gradients -> host, inside the timed region -----
+    xh, dyh = x.cpu().pin_memory(), dy.cpu().pin_memory()
+    outh = {k: torch.empty_like(v, device="cpu").pin_memory() for k, v in grads.items() if k != "dx"}
+    h2d = xh.numel() * xh.element_size() * 2
+    d2h = sum(v.numel() * v.element_size() for v in outh.values())
+
+    def e2e_step():
+        x.copy_(xh, non_blocking=True); dy.copy_(dyh, non_blocking=True)
+        step()
+        for k, v in outh.items():
+            v.copy_(grads[k], non_blocking=True)
+
+    e2e_step(); torch.cuda.synchronize()
+    barrier(); torch.cuda.synchronize()
+    e0.record()
+    for _ in range(args.steps):
+        e2e_step()
+    e1.record()
+    torch.cuda.synchronize(); barrier()
+    ms_e2e = e0.elapsed_time(e1) / args.steps
+
+    if world > 1:
+        t = torch.tensor([ms, ms_e2e], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = t.tolist()
+
+    if rank == 0:
+        peak, peak_src = measured_peaks()
+        e = 2 if w.io == "bf16" else 4
+        bytes_per_token = w.d_model * (2 * e + 4 + 2 * e) + 2 * (2 * w.d_state * 4)   # see the design doc, adjoint main kernel
+        k_ms = phase["adjoint_main"]
+        achieved = bytes_per_token * tokens / (k_ms * 1e-3) / 1e9 if k_ms > 0 else None
+        traffic = None
+        tpath = os.path.join(ROOT, "profiles", "traffic.json")
+        if os.path.exists(tpath):
+            traffic = json.load(open(tpath)).get(f"adjoint_main_kernel:{w.name}")
+        line = {"metric": METRIC, "value": world * tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": w.name, "batch": w.batch, "seq_len": w.seqlen, "d_model": w.d_model,
+                           "d_state": w.d_state, "tbar": w.tbar, "io": w.io, "layers": 1,
+                           "parallelism": "replicas only" if world > 1 else "single GPU",
+                           "l2": "inputs exceed L2 (x, dy, Delta: 0.8 GB per step)"},
+                "e2e": {"value": world * tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                        "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
+                "gpu_launches": launches,
+                "phases_ms": phase,
+                "roofline": {"kernel": "adjoint_main_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
+                             "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "traffic": traffic,
+                             "peak_source": peak_src, "bytes_per_launch": bytes_per_token * tokens,
+                             "launch_ms": k_ms},
+                "clocks": clocks}
+        if world == 1 and not args.no_cpu_baseline:
+            tps, dt, threads = oracle_sample_tokens_per_s(w, args.cpu_sample_tokens)
+            line["cpu_baseline"] = {"value": tps, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                    "sample": f"batch element 0, first {args.cpu_sample_tokens} tokens of {w.name}, "
+                                              f"Tbar={min(w.tbar, args.cpu_sample_tokens)}, all {w.d_model} channels "
+                                              f"({dt:.1f} s)"}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

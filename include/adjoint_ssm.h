@@ -1,0 +1,148 @@
+/*
+ * adjoint_ssm.h - C ABI of the B200 (sm_100a) library that computes the gradients of a diagonal
+ * selective state-space layer with the adjoint method, in full and truncated-window form.
+ *
+ * Layer (Section 3.1 "State-space models", the five steps of SSM(.), with the diagonal selective
+ * structure of Section 4.5), per sequence, t = 1..T, h_0 = 0:
+ *     Delta_t = softplus(W_delta x_t + b_delta)  [P]     B_t = W_B x_t, C_t = W_C x_t  [N]
+ *     A = -exp(A_log) [P,N]     h_t[p,n] = exp(Delta_t[p] A[p,n]) h_{t-1}[p,n] + Delta_t[p] B_t[n] x_t[p]
+ *     y_t[p] = sum_n C_t[n] h_t[p,n]
+ *
+ * Conventions for every entry point
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller, contiguous, row-major (last index
+ *     fastest) and 16-byte aligned.  Activations are [batch, seqlen, d_model]; "io dtype" is fp32 or
+ *     bf16 as selected by as_shape_t.io.  The library never allocates, frees or keeps device memory.
+ *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the legacy default
+ *     stream).  No entry point synchronises except as_check_status.
+ *   - `ws` is caller-provided scratch of at least the size reported by as_workspace_bytes; its
+ *     contents on entry are ignored and on return are unspecified.
+ *   - Return value: AS_OK (0) or a negative AS_ERR_* code.  Nothing is launched when an argument
+ *     check fails.  No exceptions, no aborts, no printing.
+ *   - Results are deterministic up to floating-point summation order (fp32 atomics are used for the
+ *     sums over channels, segments and the batch).
+ */
+#ifndef ADJOINT_SSM_H_
+#define ADJOINT_SSM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define AS_VERSION 100
+
+typedef enum { AS_F32 = 0, AS_BF16 = 1 } as_dtype_t;
+
+enum {
+  AS_OK = 0,
+  AS_ERR_NULL = -1,       /* a required pointer is NULL */
+  AS_ERR_SHAPE = -2,      /* non-positive dimension, or d_state != 16 */
+  AS_ERR_DTYPE = -3,      /* io is neither AS_F32 nor AS_BF16 */
+  AS_ERR_TBAR = -4,       /* tbar < 1 */
+  AS_ERR_WORKSPACE = -5,  /* ws_bytes smaller than as_workspace_bytes reports */
+  AS_ERR_ALIGN = -6,      /* a pointer is not 16-byte aligned, or d_model is not a multiple of 8 */
+  AS_ERR_CUDA = -7,       /* a CUDA runtime call or kernel launch failed */
+  AS_ERR_TIMEOUT = -8,    /* a bounded device-side wait gave up (reported by as_check_status) */
+  AS_ERR_LIMIT = -9       /* a size exceeds a fixed capacity of the entry point */
+};
+
+/* flags */
+#define AS_ACCUMULATE 1u  /* add into the parameter-gradient buffers instead of overwriting them */
+
+typedef struct {
+  int32_t batch;      /* Bsz >= 1 */
+  int64_t seqlen;     /* T >= 1 */
+  int32_t d_model;    /* P >= 8, multiple of 8 */
+  int32_t d_state;    /* N, must be 16 */
+  int32_t io;         /* as_dtype_t of x, y, dy, dx and the W_* matrices */
+} as_shape_t;
+
+typedef struct {          /* parameters of one layer (device pointers) */
+  const void  *W_delta;   /* [P,P] (out,in), io dtype */
+  const float *b_delta;   /* [P]   fp32 */
+  const void  *W_B;       /* [N,P] io dtype */
+  const void  *W_C;       /* [N,P] io dtype */
+  const float *A_log;     /* [P,N] fp32, A = -exp(A_log) */
+} as_params_t;
+
+typedef struct {          /* gradient outputs (device pointers); parameter gradients are fp32, summed over the batch */
+  float *dW_delta;        /* [P,P] */
+  float *db_delta;        /* [P]   */
+  float *dW_B;            /* [N,P] */
+  float *dW_C;            /* [N,P] */
+  float *dA_log;          /* [P,N] */
+  void  *dx;              /* [Bsz,T,P] io dtype, always overwritten; may be NULL (input gradient skipped) */
+} as_grads_t;
+
+/* Library version (AS_VERSION of the build). */
+int as_version(void);
+
+/* Static description of a status code. */
+const char *as_strerror(int code);
+
+/* Scratch sizes in bytes for a shape: *fwd_bytes for as_ssm_forward, *grad_bytes for as_adjoint_grad and
+ * as_full_bptt_grad (the larger of the two).  Either output pointer may be NULL.  `tbar` as for as_adjoint_grad. */
+int as_workspace_bytes(const as_shape_t *shape, int64_t tbar, size_t *fwd_bytes, size_t *grad_bytes);
+
+/* Synchronises `stream` and returns the status word the kernels keep at the start of `ws`
+ * (AS_OK, or AS_ERR_TIMEOUT if a bounded device-side wait ran out). */
+int as_check_status(const void *ws, void *stream);
+
+/* SSM(X) = Y (Section 3.1, steps 1-5; Alg. 1 line 5 for one layer).
+ * x [Bsz,T,P] io -> y [Bsz,T,P] io.  The three projections run as one dense contraction, the recurrence as
+ * a time-segmented scan (local scan per segment, sequential carry over segments, final pass). */
+int as_ssm_forward(const as_shape_t *shape, const as_params_t *params, const void *x, void *y,
+                   void *ws, size_t ws_bytes, void *stream);
+
+/* Adjoint-method gradient of L = sum_t l^t(y^t) w.r.t. the layer parameters and x, given dy = dl^t/dy^t
+ * (Proposition 2; with tbar < T the truncated form, Eq. 7 of Section 4.3; Algorithms 2-4 for one layer).
+ * Token t contributes A-net and B-net vector-Jacobian products only for source tokens i in
+ * [max(1, t+1-tbar), t]; the C-net term is never truncated.  tbar >= seqlen selects the full form.
+ * The adjoint states lambda^{t,i} are never materialised: the cotangents of all tokens t whose window
+ * contains i are summed on chip (a reverse-time recurrence with the exact removal of the term that
+ * leaves the window) and each source token's three VJPs are evaluated once.
+ * Self-contained: recomputes the forward quantities it needs from x; no prior as_ssm_forward call needed.
+ * dx also uses the windowed sum for the A/B paths and the exact C path. */
+int as_adjoint_grad(const as_shape_t *shape, const as_params_t *params, const void *x, const void *dy,
+                    int64_t tbar, uint32_t flags, const as_grads_t *out,
+                    void *ws, size_t ws_bytes, void *stream);
+
+/* The same outputs by plain backpropagation through time (the sequential nested accumulation that the
+ * adjoint method replaces, Section 3.3): one reverse sweep per channel carrying dL/dh_t.  Separately coded
+ * and deliberately simple; it exists for comparison with as_adjoint_grad at tbar >= seqlen. */
+int as_full_bptt_grad(const as_shape_t *shape, const as_params_t *params, const void *x, const void *dy,
+                      uint32_t flags, const as_grads_t *out, void *ws, size_t ws_bytes, void *stream);
+
+/* Residual-stack glue (Section 3.2; Alg. 1 lines 6-7): gain-free RMSNorm over d_model.
+ * yhat = y / sqrt(mean_p(y^2) + eps), io dtype in and out, fp32 arithmetic. */
+int as_rmsnorm_fwd(const as_shape_t *shape, const void *y, void *yhat, float eps, void *stream);
+
+/* y_out = y_in + ytilde (the residual connection y_k = y_{k-1} + SSM_k(Norm(y_{k-1}))); y_out may alias y_in. */
+int as_residual_add(const as_shape_t *shape, const void *y_in, const void *ytilde, void *y_out, void *stream);
+
+/* Backward of the glue: G_inout += RMSNormVJP(y, dyhat) = (dyhat - yhat * mean_p(dyhat*yhat)) / rms(y).
+ * G_inout [Bsz,T,P] io dtype is the upstream gradient of y (read and overwritten). */
+int as_rmsnorm_bwd_add(const as_shape_t *shape, const void *y, const void *dyhat, void *G_inout,
+                       float eps, void *stream);
+
+/* ---- diagnostics (host-side bookkeeping only; no effect on results) ------------------------------ */
+
+/* Number of kernels this library has launched in this process since the last reset; reset != 0 zeroes it. */
+int64_t as_launch_count(int reset);
+
+/* Phase timing of as_adjoint_grad.  as_set_timing(1) makes every later as_adjoint_grad call record CUDA
+ * events on its stream between its phases (this creates the events once; timing mode is opt-in and is the one
+ * place where the library creates CUDA objects).  as_get_timing synchronises on the last event of the most
+ * recent call and writes elapsed milliseconds into ms[0..AS_NUM_PHASES): projections (S1, incl. zeroing),
+ * segment pre-pass, carry fix-up, main adjoint kernel, weight-gradient contractions, input-gradient
+ * contractions.  Returns AS_OK, or AS_ERR_NULL if timing is off or no call was recorded. */
+#define AS_NUM_PHASES 6
+int as_set_timing(int enable);
+int as_get_timing(float *ms, int n);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADJOINT_SSM_H_ */

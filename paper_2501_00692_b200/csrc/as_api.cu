@@ -1,0 +1,309 @@
+// extern "C" entry points: argument checks, scratch layout, and the launch sequence of each call.
+#include <atomic>
+
+#include "as_internal.cuh"
+
+using namespace as;
+
+namespace as {
+std::atomic<int64_t> g_launches{0};
+}
+
+namespace {
+
+bool g_timing = false;
+bool g_timing_valid = false;
+cudaEvent_t g_ev[AS_NUM_PHASES + 1];
+
+void mark(int i, cudaStream_t st) {
+  if (g_timing) cudaEventRecord(g_ev[i], st);
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_shape(const as_shape_t* sh) {
+  if (!sh) return AS_ERR_NULL;
+  if (sh->batch < 1 || sh->seqlen < 1 || sh->d_model < 1) return AS_ERR_SHAPE;
+  if (sh->d_state != NS) return AS_ERR_SHAPE;
+  if (sh->io != AS_F32 && sh->io != AS_BF16) return AS_ERR_DTYPE;
+  if (sh->d_model % 8 != 0) return AS_ERR_ALIGN;
+  if (sh->batch > 65535) return AS_ERR_SHAPE;
+  return AS_OK;
+}
+
+int check_params(const as_params_t* pr) {
+  if (!pr || !pr->W_delta || !pr->b_delta || !pr->W_B || !pr->W_C || !pr->A_log) return AS_ERR_NULL;
+  if (!aligned16(pr->W_delta) || !aligned16(pr->b_delta) || !aligned16(pr->W_B) || !aligned16(pr->W_C) ||
+      !aligned16(pr->A_log))
+    return AS_ERR_ALIGN;
+  return AS_OK;
+}
+
+#define AS_TRY(expr)                      \
+  do {                                    \
+    int e__ = (expr);                     \
+    if (e__ != 0) return AS_ERR_CUDA;     \
+  } while (0)
+
+// steps 1-3 of SSM(.): Delta = softplus(x W_delta^T + b), B = x W_B^T, C = x W_C^T
+int projections(const Plan& pl, const as_params_t* pr, const void* x, char* ws, cudaStream_t st) {
+  const int bf = pl.io == AS_BF16;
+  const int64_t M = (int64_t)pl.B * pl.T;
+  GemmArgs g{};
+  g.A = x; g.a_bf16 = bf; g.a_sm = pl.P; g.a_sk = 1;
+  g.b_bf16 = bf; g.b_sn = pl.P; g.b_sk = 1;
+  g.M = M; g.K = pl.P; g.splitk = 1;
+  g.Bm = pr->W_delta; g.N = pl.P; g.C = reinterpret_cast<float*>(ws + pl.off_delta); g.ldc = pl.P; g.coff = 0;
+  g.bias = pr->b_delta; g.epi = EPI_SOFTPLUS_BIAS;
+  AS_TRY(launch_gemm_simt(g, st));
+  g.epi = EPI_STORE; g.bias = nullptr; g.N = NS; g.C = reinterpret_cast<float*>(ws + pl.off_bc); g.ldc = NBC;
+  g.Bm = pr->W_B; g.coff = 0;
+  AS_TRY(launch_gemm_simt(g, st));
+  g.Bm = pr->W_C; g.coff = NS;
+  AS_TRY(launch_gemm_simt(g, st));
+  return AS_OK;
+}
+
+int pick_splitk(int64_t tiles, int64_t K) {
+  int64_t s = (148 * 4 + tiles - 1) / tiles;
+  const int64_t maxs = (K + 255) / 256;
+  if (s > maxs) s = maxs;
+  if (s < 1) s = 1;
+  if (s > 1024) s = 1024;
+  return (int)s;
+}
+
+// the net-VJPs: weight gradients (contractions over all tokens) and the input gradient
+int contractions(const Plan& pl, const as_params_t* pr, const void* x, const as_grads_t* out, char* ws,
+                 cudaStream_t st) {
+  const int bf = pl.io == AS_BF16;
+  const int64_t M = (int64_t)pl.B * pl.T;
+  const int P = pl.P;
+  const void* du = ws + pl.off_du;
+  const float* dbc = reinterpret_cast<const float*>(ws + pl.off_dbc);
+  {  // dW_delta[i,j] = sum_m du[m,i] x[m,j]
+    GemmArgs g{};
+    g.A = du; g.a_bf16 = bf; g.a_sm = 1; g.a_sk = P;
+    g.Bm = x; g.b_bf16 = bf; g.b_sn = 1; g.b_sk = P;
+    g.C = out->dW_delta; g.ldc = P; g.coff = 0; g.M = P; g.N = P; g.K = M; g.epi = EPI_ATOMIC;
+    g.splitk = pick_splitk((int64_t)((P + 63) / 64) * ((P + 63) / 64), M);
+    AS_TRY(launch_gemm_simt(g, st));
+    // dW_B, dW_C
+    g.A = dbc; g.a_bf16 = 0; g.a_sm = 1; g.a_sk = NBC; g.M = NS;
+    g.splitk = pick_splitk((P + 63) / 64, M);
+    g.C = out->dW_B;
+    AS_TRY(launch_gemm_simt(g, st));
+    g.A = dbc + NS; g.C = out->dW_C;
+    AS_TRY(launch_gemm_simt(g, st));
+  }
+  mark(5, st);
+  if (out->dx) {  // dx = dx_dir + du W_delta + dB W_B + dC W_C
+    float* acc = reinterpret_cast<float*>(ws + pl.off_dxacc);
+    GemmArgs g{};
+    g.A = du; g.a_bf16 = bf; g.a_sm = P; g.a_sk = 1;
+    g.Bm = pr->W_delta; g.b_bf16 = bf; g.b_sn = 1; g.b_sk = P;
+    g.C = acc; g.ldc = P; g.coff = 0; g.M = M; g.N = P; g.K = P; g.epi = EPI_STORE; g.splitk = 1;
+    AS_TRY(launch_gemm_simt(g, st));
+    g.A = dbc; g.a_bf16 = 0; g.a_sm = NBC; g.a_sk = 1; g.K = NS; g.epi = EPI_ACCUM;
+    g.Bm = pr->W_B;
+    AS_TRY(launch_gemm_simt(g, st));
+    g.A = dbc + NS; g.Bm = pr->W_C;
+    AS_TRY(launch_gemm_simt(g, st));
+    AS_TRY(launch_finish_dx(pl, acc, ws + pl.off_dxdir, out->dx, st));
+  }
+  mark(6, st);
+  return AS_OK;
+}
+
+int check_grad_args(const as_shape_t* sh, const as_params_t* pr, const void* x, const void* dy,
+                    const as_grads_t* out, void* ws) {
+  int e = check_shape(sh);
+  if (e) return e;
+  e = check_params(pr);
+  if (e) return e;
+  if (!x || !dy || !out || !ws) return AS_ERR_NULL;
+  if (!out->dW_delta || !out->db_delta || !out->dW_B || !out->dW_C || !out->dA_log) return AS_ERR_NULL;
+  if (!aligned16(x) || !aligned16(dy) || !aligned16(ws) || !aligned16(out->dW_delta) || !aligned16(out->db_delta) ||
+      !aligned16(out->dW_B) || !aligned16(out->dW_C) || !aligned16(out->dA_log) || !aligned16(out->dx))
+    return AS_ERR_ALIGN;
+  return AS_OK;
+}
+
+int zero_outputs(const Plan& pl, uint32_t flags, const as_grads_t* out, char* ws, cudaStream_t st) {
+  const size_t P = pl.P;
+  AS_TRY((int)cudaMemsetAsync(ws + pl.off_status, 0, 256, st));
+  AS_TRY((int)cudaMemsetAsync(ws + pl.off_dbc, 0, (size_t)pl.B * pl.T * NBC * 4, st));
+  if (!(flags & AS_ACCUMULATE)) {
+    AS_TRY((int)cudaMemsetAsync(out->dW_delta, 0, P * P * 4, st));
+    AS_TRY((int)cudaMemsetAsync(out->db_delta, 0, P * 4, st));
+    AS_TRY((int)cudaMemsetAsync(out->dW_B, 0, NS * P * 4, st));
+    AS_TRY((int)cudaMemsetAsync(out->dW_C, 0, NS * P * 4, st));
+    AS_TRY((int)cudaMemsetAsync(out->dA_log, 0, P * NS * 4, st));
+  }
+  return AS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int as_version(void) { return AS_VERSION; }
+
+const char* as_strerror(int code) {
+  switch (code) {
+    case AS_OK: return "ok";
+    case AS_ERR_NULL: return "a required pointer is NULL";
+    case AS_ERR_SHAPE: return "bad shape (non-positive dimension or d_state != 16)";
+    case AS_ERR_DTYPE: return "unsupported io dtype";
+    case AS_ERR_TBAR: return "tbar must be >= 1";
+    case AS_ERR_WORKSPACE: return "workspace too small";
+    case AS_ERR_ALIGN: return "pointer not 16-byte aligned or d_model not a multiple of 8";
+    case AS_ERR_CUDA: return "CUDA runtime call or launch failed";
+    case AS_ERR_TIMEOUT: return "bounded device-side wait gave up";
+    case AS_ERR_LIMIT: return "size exceeds a fixed capacity of this entry point";
+    default: return "unknown status code";
+  }
+}
+
+int as_workspace_bytes(const as_shape_t* shape, int64_t tbar, size_t* fwd_bytes, size_t* grad_bytes) {
+  int e = check_shape(shape);
+  if (e) return e;
+  if (tbar < 1) return AS_ERR_TBAR;
+  Plan pl;
+  make_plan(shape, tbar, &pl);
+  if (fwd_bytes) *fwd_bytes = pl.total_fwd;
+  if (grad_bytes) *grad_bytes = pl.total_grad;
+  return AS_OK;
+}
+
+int as_check_status(const void* ws, void* stream) {
+  if (!ws) return AS_ERR_NULL;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  int word = 0;
+  if (cudaMemcpyAsync(&word, ws, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return AS_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return AS_ERR_CUDA;
+  return word;
+}
+
+int as_ssm_forward(const as_shape_t* shape, const as_params_t* params, const void* x, void* y, void* ws,
+                   size_t ws_bytes, void* stream) {
+  int e = check_shape(shape);
+  if (e) return e;
+  e = check_params(params);
+  if (e) return e;
+  if (!x || !y || !ws) return AS_ERR_NULL;
+  if (!aligned16(x) || !aligned16(y) || !aligned16(ws)) return AS_ERR_ALIGN;
+  Plan pl;
+  make_plan(shape, shape->seqlen, &pl);
+  if (ws_bytes < pl.total_fwd) return AS_ERR_WORKSPACE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  char* w = reinterpret_cast<char*>(ws);
+  AS_TRY((int)cudaMemsetAsync(w + pl.off_status, 0, 256, st));
+  e = projections(pl, params, x, w, st);
+  if (e) return e;
+  ScanPtrs sp{x, nullptr, params->A_log, w};
+  AS_TRY(launch_prepass(pl, sp, false, false, st));
+  AS_TRY(launch_fixup(pl, sp, false, st));
+  AS_TRY(launch_forward_y(pl, sp, y, st));
+  return AS_OK;
+}
+
+int as_adjoint_grad(const as_shape_t* shape, const as_params_t* params, const void* x, const void* dy, int64_t tbar,
+                    uint32_t flags, const as_grads_t* out, void* ws, size_t ws_bytes, void* stream) {
+  int e = check_grad_args(shape, params, x, dy, out, ws);
+  if (e) return e;
+  if (tbar < 1) return AS_ERR_TBAR;
+  Plan pl;
+  make_plan(shape, tbar, &pl);
+  if (ws_bytes < pl.total_grad) return AS_ERR_WORKSPACE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  char* w = reinterpret_cast<char*>(ws);
+  mark(0, st);
+  e = zero_outputs(pl, flags, out, w, st);
+  if (e) return e;
+  e = projections(pl, params, x, w, st);
+  if (e) return e;
+  mark(1, st);
+  ScanPtrs sp{x, dy, params->A_log, w};
+  AS_TRY(launch_prepass(pl, sp, true, true, st));
+  mark(2, st);
+  AS_TRY(launch_fixup(pl, sp, true, st));
+  mark(3, st);
+  AS_TRY(launch_adjoint_main(pl, sp, out->dA_log, out->db_delta, st));
+  mark(4, st);
+  e = contractions(pl, params, x, out, w, st);
+  if (g_timing && e == AS_OK) g_timing_valid = true;
+  return e;
+}
+
+int as_full_bptt_grad(const as_shape_t* shape, const as_params_t* params, const void* x, const void* dy,
+                      uint32_t flags, const as_grads_t* out, void* ws, size_t ws_bytes, void* stream) {
+  int e = check_grad_args(shape, params, x, dy, out, ws);
+  if (e) return e;
+  Plan pl;
+  make_plan(shape, shape->seqlen, &pl);
+  if (ws_bytes < pl.total_grad) return AS_ERR_WORKSPACE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  char* w = reinterpret_cast<char*>(ws);
+  e = zero_outputs(pl, flags, out, w, st);
+  if (e) return e;
+  e = projections(pl, params, x, w, st);
+  if (e) return e;
+  ScanPtrs sp{x, dy, params->A_log, w};
+  AS_TRY(launch_bptt(pl, sp, out->dA_log, out->db_delta, st));
+  return contractions(pl, params, x, out, w, st);
+}
+
+int as_rmsnorm_fwd(const as_shape_t* shape, const void* y, void* yhat, float eps, void* stream) {
+  int e = check_shape(shape);
+  if (e) return e;
+  if (!y || !yhat) return AS_ERR_NULL;
+  AS_TRY(launch_rmsnorm_fwd(shape, y, yhat, eps, reinterpret_cast<cudaStream_t>(stream)));
+  return AS_OK;
+}
+
+int as_residual_add(const as_shape_t* shape, const void* y_in, const void* ytilde, void* y_out, void* stream) {
+  int e = check_shape(shape);
+  if (e) return e;
+  if (!y_in || !ytilde || !y_out) return AS_ERR_NULL;
+  AS_TRY(launch_residual_add(shape, y_in, ytilde, y_out, reinterpret_cast<cudaStream_t>(stream)));
+  return AS_OK;
+}
+
+int as_rmsnorm_bwd_add(const as_shape_t* shape, const void* y, const void* dyhat, void* G_inout, float eps,
+                       void* stream) {
+  int e = check_shape(shape);
+  if (e) return e;
+  if (!y || !dyhat || !G_inout) return AS_ERR_NULL;
+  AS_TRY(launch_rmsnorm_bwd_add(shape, y, dyhat, G_inout, eps, reinterpret_cast<cudaStream_t>(stream)));
+  return AS_OK;
+}
+
+int64_t as_launch_count(int reset) {
+  const int64_t v = as::g_launches.load();
+  if (reset) as::g_launches.store(0);
+  return v;
+}
+
+int as_set_timing(int enable) {
+  static bool created = false;
+  if (enable && !created) {
+    for (int i = 0; i <= AS_NUM_PHASES; ++i)
+      if (cudaEventCreate(&g_ev[i]) != cudaSuccess) return AS_ERR_CUDA;
+    created = true;
+  }
+  g_timing = enable != 0;
+  g_timing_valid = false;
+  return AS_OK;
+}
+
+int as_get_timing(float* ms, int n) {
+  if (!ms) return AS_ERR_NULL;
+  if (!g_timing || !g_timing_valid) return AS_ERR_NULL;
+  if (cudaEventSynchronize(g_ev[AS_NUM_PHASES]) != cudaSuccess) return AS_ERR_CUDA;
+  for (int i = 0; i < n && i < AS_NUM_PHASES; ++i)
+    if (cudaEventElapsedTime(&ms[i], g_ev[i], g_ev[i + 1]) != cudaSuccess) return AS_ERR_CUDA;
+  return AS_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,98 @@
+// Internal declarations shared by the translation units of libadjoint_ssm (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include <atomic>
+
+#include "../../include/adjoint_ssm.h"
+
+namespace as {
+
+extern std::atomic<int64_t> g_launches;   // kernels launched by this library (diagnostic)
+inline void count_launch(int n = 1) { g_launches.fetch_add(n); }
+
+constexpr int NS = 16;        // d_state handled by the scan kernels
+constexpr int CK = 8;         // tokens per checkpoint chunk (h of one chunk lives in registers)
+constexpr int CH = 128;       // channels per CTA of the scan kernels
+constexpr int NBC = 2 * NS;   // per-token row of [B_t | C_t] (and of [dB_t | dC_t])
+constexpr float LOG2E = 1.4426950408889634f;
+constexpr float LN2 = 0.6931471805599453f;
+
+// ---- I/O element access ---------------------------------------------------------------------
+template <typename T> __device__ __forceinline__ float ld_io(const T* p);
+template <> __device__ __forceinline__ float ld_io<float>(const float* p) { return __ldg(p); }
+template <> __device__ __forceinline__ float ld_io<__nv_bfloat16>(const __nv_bfloat16* p) {
+  return __bfloat162float(__ldg(p));
+}
+template <typename T> __device__ __forceinline__ void st_io(T* p, float v);
+template <> __device__ __forceinline__ void st_io<float>(float* p, float v) { *p = v; }
+template <> __device__ __forceinline__ void st_io<__nv_bfloat16>(__nv_bfloat16* p, float v) {
+  *p = __float2bfloat16_rn(v);
+}
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// ---- time segmentation and scratch layout ---------------------------------------------------
+// Time is cut into S segments of L tokens (L a multiple of CK); a CTA owns (segment, batch element,
+// CH channels).  Per-(segment, channel, state) arrays use the float4-friendly order [.., 4, P, 4]
+// (state n = 4*q + r lives at ((q*P + p)*4 + r)) so that a warp's accesses are contiguous.
+struct Plan {
+  int B, P;
+  int64_t T;
+  int64_t tbar;     // clamped to T
+  int full;         // tbar >= T
+  int L;            // segment length (tokens)
+  int S;            // number of segments
+  int64_t NC;       // number of CK-token chunks = ceil(T/CK)
+  int m;            // tbar / L   (whole segments inside a window that starts on a segment boundary)
+  int r;            // tbar % L   (tokens of the following partial segment)
+  int io;           // as_dtype_t
+  // byte offsets into the workspace
+  size_t off_status, off_delta, off_bc, off_ckpt, off_cs, off_hend, off_muloc, off_mupart, off_segd,
+      off_partd, off_firstd, off_hstart, off_carry, off_swin, off_du, off_dxdir, off_dbc, off_dxacc,
+      off_bptt_ckpt, total_fwd, total_grad;
+};
+
+int make_plan(const as_shape_t* sh, int64_t tbar, Plan* pl);
+
+// ---- launchers (each returns a cudaError_t as int) ------------------------------------------
+// C[m, coff + n] (ldc) = epi( sum_k A(m,k) B(n,k) ), fp32 accumulation on the FP32 pipe.
+enum { EPI_STORE = 0, EPI_SOFTPLUS_BIAS = 1, EPI_ATOMIC = 2, EPI_ACCUM = 3 };
+struct GemmArgs {
+  const void* A; int a_bf16; int64_t a_sm, a_sk;   // element strides of A(m,k)
+  const void* Bm; int b_bf16; int64_t b_sn, b_sk;  // element strides of B(n,k)
+  float* C; int64_t ldc; int64_t coff;
+  const float* bias;
+  int64_t M; int N; int64_t K;
+  int epi;
+  int splitk;                                      // >1 only with EPI_ATOMIC
+};
+int launch_gemm_simt(const GemmArgs& g, cudaStream_t st);
+
+struct ScanPtrs {
+  const void *x, *dy;
+  const float* A_log;
+  char* ws;
+};
+int launch_prepass(const Plan& pl, const ScanPtrs& sp, bool with_mu, bool with_ckpt, cudaStream_t st);
+int launch_fixup(const Plan& pl, const ScanPtrs& sp, bool with_mu, cudaStream_t st);
+int launch_forward_y(const Plan& pl, const ScanPtrs& sp, void* y, cudaStream_t st);
+int launch_adjoint_main(const Plan& pl, const ScanPtrs& sp, float* dA_log, float* db_delta, cudaStream_t st);
+int launch_finish_dx(const Plan& pl, const float* dxacc, const void* dxdir, void* dx, cudaStream_t st);
+
+int launch_bptt(const Plan& pl, const ScanPtrs& sp, float* dA_log, float* db_delta, cudaStream_t st);
+
+int launch_rmsnorm_fwd(const as_shape_t* sh, const void* y, void* yhat, float eps, cudaStream_t st);
+int launch_residual_add(const as_shape_t* sh, const void* a, const void* b, void* out, cudaStream_t st);
+int launch_rmsnorm_bwd_add(const as_shape_t* sh, const void* y, const void* dyhat, void* G, float eps,
+                           cudaStream_t st);
+
+}  // namespace as

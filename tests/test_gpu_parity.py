@@ -1,0 +1,125 @@
+"""CUDA path vs the fp64 oracle, element by element, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ssm_oracle as O
+from paper_2501_00692_b200 import binding as B
+from paper_2501_00692_b200 import synth
+from paper_2501_00692_b200.build import build_library
+
+from gpu_util import (TOL, assert_close, compare_grads, gpu_adjoint, gpu_forward, oracle_adjoint, theta_f64)
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build_library()
+    B.lib()
+
+
+def setup(w, slow=False, layer=0):
+    theta = synth.layer_params(w, layer, DEV, slow_decay=slow)
+    x, dy = synth.activations(w, DEV)
+    return theta, x, dy
+
+
+def test_c1_forward_and_full_adjoint_fp32():
+    w = synth.WORKLOADS["C1"]
+    theta, x, dy = setup(w)
+    y = gpu_forward(w, theta, x)
+    yref = np.stack([O.ssm_forward(theta_f64(theta), synth.to_f64(x)[b]) for b in range(w.batch)])
+    assert_close(synth.to_f64(y), yref, TOL["f32"], "y")
+    ref = oracle_adjoint(theta, x, dy, w.tbar, tier="direct")
+    compare_grads(gpu_adjoint(w, theta, x, dy, w.tbar), ref, TOL["f32"])
+    # truncated == full once the window covers the sequence (Eq. 7), on the GPU too
+    compare_grads(gpu_adjoint(w, theta, x, dy, w.seqlen + 5), ref, TOL["f32"])
+
+
+def test_c1_bptt_comparator_matches_oracle_and_adjoint():
+    w = synth.WORKLOADS["C1"]
+    theta, x, dy = setup(w)
+    th = theta_f64(theta)
+    ref = O.batched(O.bptt_grad, th, synth.to_f64(x), synth.to_f64(dy))
+    gb = gpu_adjoint(w, theta, x, dy, w.tbar, bptt=True)
+    compare_grads(gb, ref, TOL["f32"])
+    ga = gpu_adjoint(w, theta, x, dy, w.tbar)
+    for k in O.PARAM_GRADS + ("dx",):
+        assert_close(synth.to_f64(ga[k]), synth.to_f64(gb[k]), TOL["f32"], "adjoint vs bptt " + k)
+
+
+@pytest.mark.parametrize("slow", [False, True])
+@pytest.mark.parametrize("tbar", [1, 2, 7, 8, 9, 63, 64, 65, 127, 128, 129, 200, 299, 300, 301])
+def test_ragged_small_shapes_window_edges(tbar, slow):
+    # several 64-token segments with a ragged last one, d_model not a multiple of the warp width,
+    # windows below / at / above segment multiples
+    w = synth.custom_workload("ragged", 11, 2, 300, 40, tbar=tbar, io="f32")
+    theta, x, dy = setup(w, slow)
+    ref = oracle_adjoint(theta, x, dy, tbar, tier="direct")
+    compare_grads(gpu_adjoint(w, theta, x, dy, tbar), ref, TOL["f32"])
+
+
+def test_impulse_window_edges_on_gpu():
+    # upstream gradient = one impulse: B-path outputs are non-zero exactly on the window (Eq. 7 ranges)
+    w = synth.custom_workload("impulse", 12, 1, 200, 32, tbar=70, io="f32")
+    theta, x, dy = setup(w, slow=True)
+    dy.zero_()
+    tp, pp = 150, 5
+    dy[0, tp, pp] = 1.0
+    g = gpu_adjoint(w, theta, x, dy, w.tbar)
+    ref = oracle_adjoint(theta, x, dy, w.tbar, tier="direct")
+    compare_grads(g, ref, TOL["f32"])
+    # dx = dx_dir + (dense parts); the dense parts vanish where du, dB, dC vanish: rows outside the window are 0
+    dx = synth.to_f64(g["dx"])[0]
+    nz = np.abs(dx).max(axis=1) > 0
+    want = np.zeros(w.seqlen, bool); want[tp - w.tbar + 1:tp + 1] = True
+    assert (nz == want).all()
+
+
+def test_accumulate_flag_and_no_dx():
+    w = synth.custom_workload("acc", 13, 1, 128, 32, tbar=20, io="f32")
+    theta, x, dy = setup(w)
+    g1 = gpu_adjoint(w, theta, x, dy, w.tbar)
+    g2 = gpu_adjoint(w, theta, x, dy, w.tbar, with_dx=False)
+    g2 = gpu_adjoint(w, theta, x, dy, w.tbar, flags=B.AS_ACCUMULATE, grads=g2, with_dx=False)
+    for k in O.PARAM_GRADS:
+        assert_close(synth.to_f64(g2[k]), 2 * synth.to_f64(g1[k]), 1e-5, k)
+
+
+def test_c2_truncated_and_full_fp32():
+    w = synth.WORKLOADS["C2"]
+    for slow in (False, True):
+        theta, x, dy = setup(w, slow)
+        ref = oracle_adjoint(theta, x, dy, w.tbar, tier="direct")       # Tbar = 64: the defining double sum
+        compare_grads(gpu_adjoint(w, theta, x, dy, w.tbar), ref, TOL["f32"])
+        full = oracle_adjoint(theta, x, dy, w.seqlen, tier="block")
+        compare_grads(gpu_adjoint(w, theta, x, dy, w.seqlen), full, TOL["f32"])
+        if slow:   # the window is visible: truncated and full differ by far more than the tolerance
+            assert np.abs(ref["dW_B"] - full["dW_B"]).max() / np.abs(full["dW_B"]).max() > 1e-2
+
+
+@pytest.mark.parametrize("slow", [False, True])
+def test_bf16_multi_segment(slow):
+    w = synth.custom_workload("bf16", 14, 2, 4096, 128, tbar=1000, io="bf16")
+    theta, x, dy = setup(w, slow)
+    ref = oracle_adjoint(theta, x, dy, w.tbar, tier="block")
+    compare_grads(gpu_adjoint(w, theta, x, dy, w.tbar), ref, TOL["bf16"])
+    y = gpu_forward(w, theta, x)
+    assert_close(synth.to_f64(y), ref["y"], TOL["bf16"], "y")
+
+
+def test_rmsnorm_glue():
+    w = synth.custom_workload("norm", 15, 2, 33, 72, io="f32")
+    _, y, d = setup(w)
+    sh = B.shape_of(y)
+    yhat = torch.empty_like(y)
+    B.as_rmsnorm_fwd(sh, y, yhat)
+    assert_close(synth.to_f64(yhat), O.rmsnorm(synth.to_f64(y)), 1e-5, "rmsnorm")
+    G = d.clone()
+    B.as_rmsnorm_bwd_add(sh, y, d, G)
+    assert_close(synth.to_f64(G), synth.to_f64(d) + O.rmsnorm_vjp(synth.to_f64(y), synth.to_f64(d)), 1e-5, "rmsnorm vjp")
+    out = torch.empty_like(y)
+    B.as_residual_add(sh, y, d, out)
+    assert torch.equal(out, y + d)
