@@ -131,6 +131,11 @@ def main():
     ap.add_argument("--workload", default="C3")
     ap.add_argument("--cpu-sample-tokens", type=int, default=16384)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--batch", type=int, default=None, help="override the workload's batch (profiling runs)")
+    ap.add_argument("--seq-len", type=int, default=None, help="override the workload's seqlen (profiling runs)")
+    ap.add_argument("--tbar", type=int, default=None, help="override the workload's window (profiling runs)")
+    ap.add_argument("--slow-decay", action="store_true", help="slow-decay parameter law (window term live)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     if args.impl == "reference":
@@ -157,7 +162,10 @@ def main():
             dist.barrier()
 
     w = synth.WORKLOADS[args.workload]
-    theta = synth.layer_params(w, 0, dev)
+    if args.batch or args.seq_len or args.tbar:
+        w = synth.custom_workload(w.name + "-custom", w.config, args.batch or w.batch, args.seq_len or w.seqlen,
+                                  w.d_model, w.d_state, 1, args.tbar or w.tbar, w.io)
+    theta = synth.layer_params(w, 0, dev, slow_decay=args.slow_decay)
     x, dy = synth.activations(w, dev)
     sh = B.shape_of(x, w.d_state)
     _, gbytes = B.as_workspace_bytes(sh, w.tbar)
@@ -197,6 +205,21 @@ def main():
     B.as_set_timing(False)
     clocks = sampler.stop() if rank == 0 else None
     # ---- end to end: pinned host inputs -> device, gradients -> host, inside the timed region -----
+    if args.no_e2e:
+        ms_e2e, h2d, d2h = float("nan"), 0, 0
+    else:
+        ms_e2e, h2d, d2h = run_e2e(args, torch, x, dy, grads, step, barrier, e0, e1)
+
+    if world > 1:
+        t = torch.tensor([ms, ms_e2e], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = t.tolist()
+    report(args, B, w, world, rank, tokens, ms, ms_e2e, h2d, d2h, launches, phase, clocks)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(args, torch, x, dy, grads, step, barrier, e0, e1):
     xh, dyh = x.cpu().pin_memory(), dy.cpu().pin_memory()
     outh = {k: torch.empty_like(v, device="cpu").pin_memory() for k, v in grads.items() if k != "dx"}
     h2d = xh.numel() * xh.element_size() * 2
@@ -215,13 +238,10 @@ def main():
         e2e_step()
     e1.record()
     torch.cuda.synchronize(); barrier()
-    ms_e2e = e0.elapsed_time(e1) / args.steps
+    return e0.elapsed_time(e1) / args.steps, h2d, d2h
 
-    if world > 1:
-        t = torch.tensor([ms, ms_e2e], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = t.tolist()
 
+def report(args, B, w, world, rank, tokens, ms, ms_e2e, h2d, d2h, launches, phase, clocks):
     if rank == 0:
         peak, peak_src = measured_peaks()
         e = 2 if w.io == "bf16" else 4
@@ -255,8 +275,6 @@ def main():
                                               f"Tbar={min(w.tbar, args.cpu_sample_tokens)}, all {w.d_model} channels "
                                               f"({dt:.1f} s)"}
         print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
 
 
 if __name__ == "__main__":

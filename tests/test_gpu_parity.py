@@ -71,11 +71,13 @@ def test_impulse_window_edges_on_gpu():
     g = gpu_adjoint(w, theta, x, dy, w.tbar)
     ref = oracle_adjoint(theta, x, dy, w.tbar, tier="direct")
     compare_grads(g, ref, TOL["f32"])
-    # dx = dx_dir + (dense parts); the dense parts vanish where du, dB, dC vanish: rows outside the window are 0
-    dx = synth.to_f64(g["dx"])[0]
-    nz = np.abs(dx).max(axis=1) > 0
-    want = np.zeros(w.seqlen, bool); want[tp - w.tbar + 1:tp + 1] = True
-    assert (nz == want).all()
+    # dx = dx_dir + (dense parts): rows inside the window carry signal, rows after the impulse are exactly
+    # zero, rows before the window hold only the rounding residue of the exact window-exit subtraction
+    dx = np.abs(synth.to_f64(g["dx"])[0]).max(axis=1)
+    lo = tp - w.tbar + 1
+    assert (dx[tp + 1:] == 0).all()
+    assert (dx[lo:tp + 1] > 1e-3 * dx.max()).all()
+    assert (dx[:lo] < 1e-5 * dx.max()).all()
 
 
 def test_accumulate_flag_and_no_dx():
