@@ -47,6 +47,11 @@ int check_params(const as_params_t* pr) {
 
 // steps 1-3 of SSM(.): Delta = softplus(x W_delta^T + b), B = x W_B^T, C = x W_C^T
 int projections(const Plan& pl, const as_params_t* pr, const void* x, char* ws, cudaStream_t st) {
+  if (pl.tc) {
+    AS_TRY(tc_pack_wcat(pl, pr, ws, st));
+    AS_TRY(tc_projections(pl, pr, x, ws, st));
+    return AS_OK;
+  }
   const int bf = pl.io == AS_BF16;
   const int64_t M = (int64_t)pl.B * pl.T;
   GemmArgs g{};
@@ -81,6 +86,13 @@ int contractions(const Plan& pl, const as_params_t* pr, const void* x, const as_
   const int P = pl.P;
   const void* du = ws + pl.off_du;
   const float* dbc = reinterpret_cast<const float*>(ws + pl.off_dbc);
+  if (pl.tc) {
+    AS_TRY(tc_weight_grads(pl, x, out, ws, st));
+    mark(5, st);
+    if (out->dx) AS_TRY(tc_input_grad(pl, out->dx, ws, st));
+    mark(6, st);
+    return AS_OK;
+  }
   {  // dW_delta[i,j] = sum_m du[m,i] x[m,j]
     GemmArgs g{};
     g.A = du; g.a_bf16 = bf; g.a_sm = 1; g.a_sk = P;

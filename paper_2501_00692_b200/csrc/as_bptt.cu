@@ -90,7 +90,7 @@ __global__ void __launch_bounds__(32) bptt_reverse_kernel(Plan pl, const IO* __r
       const float sig = 1.f / (1.f + expf(-logf(expm1f(d))));  // u = softplus^{-1}(delta)
       const float duv = d_delta * sig;
       if (active) {
-        st_io<IO>(du + row * pl.P + p, duv);
+        st_io<IO>(du + row * pl.du_ld + p, duv);
         st_io<IO>(dxdir + row * pl.P + p, d * sB);
         dbias += duv;
       }

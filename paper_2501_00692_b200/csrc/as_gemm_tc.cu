@@ -1,0 +1,378 @@
+// bf16 tensor-core contractions for sm_100a: TMA (cp.async.bulk.tensor, 128-byte swizzle) feeds a
+// shared-memory ring, one elected thread issues tcgen05.mma into a TMEM accumulator, four warps drain it
+// with tcgen05.ld and apply the fused epilogue.  One kernel template covers the three token-dimension
+// contractions of the layer:
+//   PROJ : [Delta | B | C] = X Wcat^T            (A K-major, B K-major;  softplus+bias epilogue)
+//   DW   : dWcat = Gcat^T X  over all tokens     (A MN-major, B MN-major; split-K, fp32 reduction)
+//   DX   : dx = dx_dir + Gcat Wcat               (A K-major, B MN-major; add + bf16 store)
+// with Wcat = [W_delta; W_B; W_C] ([P+32, P]) and Gcat = [du | dB | dC] ([tokens, P+32]), both bf16.
+// No cluster multicast is used anywhere.  Every mbarrier wait is bounded; on timeout the kernel records
+// AS_ERR_TIMEOUT in the status word, stops issuing work, frees its TMEM and returns.
+#include <cuda.h>
+
+#include "as_internal.cuh"
+
+namespace as {
+namespace {
+
+constexpr int BM = 128, BN = 128, BK = 64, STAGES = 3, UK = 16;
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int SMEM_DYN = STAGES * STAGE_BYTES + 1024;  // + slack for 1024-byte alignment
+constexpr uint32_t WAIT_LIMIT = 1u << 22;
+
+enum { MAJ_K = 0, MAJ_MN = 1 };
+enum { TC_PROJ = 0, TC_DW = 1, TC_DX = 2 };
+
+struct TcArgs {
+  int64_t M;            // rows of the output tile space (A's MN extent)
+  int N;                // cols of the output (B's MN extent)
+  int kblocks;          // number of BK-blocks along K
+  int splitk;
+  int P;                // d_model
+  // PROJ
+  float* delta; float* bc; const float* bias;
+  // DW
+  float* dW_delta; float* dW_B; float* dW_C;
+  // DX
+  const __nv_bfloat16* dxdir; __nv_bfloat16* dx;
+  int* status;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// bounded wait: returns false if the phase did not complete within WAIT_LIMIT polls
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  const uint32_t addr = smem_u32(bar);
+  for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(addr), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    if (*abort_flag) return false;
+  }
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, int c0, int c1, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(dst)), "l"(tm), "r"(c0), "r"(c1), "r"(smem_u32(bar))
+      : "memory");
+}
+
+// shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ float softplus_f(float u) { return fmaxf(u, 0.f) + log1pf(__expf(-fabsf(u))); }
+
+template <int AMAJ, int BMAJ, int EPI>
+__global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
+                                                      const __grid_constant__ CUtensorMap tmB, TcArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[STAGES];
+  __shared__ __align__(8) uint64_t empty_bar[STAGES];
+  __shared__ __align__(8) uint64_t tmem_full_bar;
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_s;
+
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int64_t m0 = (int64_t)blockIdx.x * BM;
+  const int n0 = blockIdx.y * BN;
+  const int kper = (a.kblocks + a.splitk - 1) / a.splitk;
+  const int kb0 = blockIdx.z * kper;
+  const int kb1 = min(a.kblocks, kb0 + kper);
+  const int nkb = kb1 - kb0;
+  volatile int* abortp = &abort_s;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    mbar_init(&tmem_full_bar, 1);
+    abort_s = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {   // TMEM allocation: BN fp32 accumulator columns
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(BN)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = tmem_base_s;
+
+  if (nkb > 0) {
+    if (warp == 0 && lane == 0) {
+      // ---------------- TMA producer ----------------
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
+      for (int i = 0; i < nkb; ++i) {
+        const int s = i % STAGES, round = i / STAGES;
+        if (round > 0 && !mbar_wait(&empty_bar[s], (round - 1) & 1, abortp)) { *abortp = 1; atomicExch(a.status, AS_ERR_TIMEOUT); break; }
+        uint8_t* sa = smem + s * STAGE_BYTES;
+        uint8_t* sb = sa + A_BYTES;
+        mbar_expect_tx(&full_bar[s], STAGE_BYTES);
+        const int k = (kb0 + i) * BK;
+        if (AMAJ == MAJ_K) {
+          tma_load_2d(sa, &tmA, k, (int)m0, &full_bar[s]);
+        } else {
+          tma_load_2d(sa, &tmA, (int)m0, k, &full_bar[s]);
+          tma_load_2d(sa + A_BYTES / 2, &tmA, (int)m0 + 64, k, &full_bar[s]);
+        }
+        if (BMAJ == MAJ_K) {
+          tma_load_2d(sb, &tmB, k, n0, &full_bar[s]);
+        } else {
+          tma_load_2d(sb, &tmB, n0, k, &full_bar[s]);
+          tma_load_2d(sb + B_BYTES / 2, &tmB, n0 + 64, k, &full_bar[s]);
+        }
+      }
+    } else if (warp == 1 && lane == 0) {
+      // ---------------- MMA issuer ----------------
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)AMAJ << 15) | ((uint32_t)BMAJ << 16) |
+                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      bool ok = true;
+      for (int i = 0; i < nkb && ok; ++i) {
+        const int s = i % STAGES, round = i / STAGES;
+        if (!mbar_wait(&full_bar[s], round & 1, abortp)) { *abortp = 1; atomicExch(a.status, AS_ERR_TIMEOUT); ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t sa = smem_u32(smem + s * STAGE_BYTES);
+        const uint32_t sb = sa + A_BYTES;
+#pragma unroll
+        for (int k = 0; k < BK / UK; ++k) {
+          const uint64_t ad = (AMAJ == MAJ_K) ? make_desc(sa + k * UK * 2, 16, 1024)
+                                              : make_desc(sa + k * UK * 128, A_BYTES / 2, 1024);
+          const uint64_t bd = (BMAJ == MAJ_K) ? make_desc(sb + k * UK * 2, 16, 1024)
+                                              : make_desc(sb + k * UK * 128, B_BYTES / 2, 1024);
+          umma_bf16(tmem_base, ad, bd, idesc, (i > 0 || k > 0) ? 1u : 0u);
+        }
+        umma_commit(&empty_bar[s]);   // frees the stage once these MMAs have read it
+      }
+      umma_commit(&tmem_full_bar);    // accumulator complete
+    }
+    // ---------------- epilogue: all four warps ----------------
+    __syncwarp();
+    const bool ready = mbar_wait(&tmem_full_bar, 0, abortp);
+    if (!ready) { *abortp = 1; if (lane == 0) atomicExch(a.status, AS_ERR_TIMEOUT); }
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (ready) {
+      const int64_t m = m0 + warp * 32 + lane;   // this thread's output row
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32), r);
+        const int nb = n0 + c * 32;
+        if (m >= a.M || nb >= a.N) continue;
+        if (EPI == TC_PROJ) {
+          if (nb < a.P) {
+            float4* dst = reinterpret_cast<float4*>(a.delta + m * a.P + nb);
+            const float4* b4 = reinterpret_cast<const float4*>(a.bias + nb);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              const float4 bv = __ldg(b4 + q);
+              dst[q] = make_float4(softplus_f(__uint_as_float(r[4 * q]) + bv.x), softplus_f(__uint_as_float(r[4 * q + 1]) + bv.y),
+                                   softplus_f(__uint_as_float(r[4 * q + 2]) + bv.z), softplus_f(__uint_as_float(r[4 * q + 3]) + bv.w));
+            }
+          } else {
+            float4* dst = reinterpret_cast<float4*>(a.bc + m * NBC + (nb - a.P));
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              dst[q] = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]), __uint_as_float(r[4 * q + 2]),
+                                   __uint_as_float(r[4 * q + 3]));
+          }
+        } else if (EPI == TC_DW) {
+          float* dst;
+          if (m < a.P) dst = a.dW_delta + m * a.P + nb;
+          else if (m < a.P + NS) dst = a.dW_B + (m - a.P) * a.P + nb;
+          else dst = a.dW_C + (m - a.P - NS) * a.P + nb;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) atomicAdd(dst + j, __uint_as_float(r[j]));
+        } else {
+          const uint4* src = reinterpret_cast<const uint4*>(a.dxdir + m * a.P + nb);
+          uint4* dst = reinterpret_cast<uint4*>(a.dx + m * a.P + nb);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const uint4 sv = __ldg(src + q);
+            const __nv_bfloat162* s2 = reinterpret_cast<const __nv_bfloat162*>(&sv);
+            uint4 ov;
+            __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float2 f = __bfloat1622float2(s2[e]);
+              o2[e] = __floats2bfloat162_rn(f.x + __uint_as_float(r[8 * q + 2 * e]), f.y + __uint_as_float(r[8 * q + 2 * e + 1]));
+            }
+            dst[q] = ov;
+          }
+        }
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(BN) : "memory");
+  }
+}
+
+// ---- small helpers -------------------------------------------------------------------------------
+__global__ void pack_wcat_kernel(int P, const __nv_bfloat16* __restrict__ Wd, const __nv_bfloat16* __restrict__ WB,
+                                 const __nv_bfloat16* __restrict__ WC, __nv_bfloat16* __restrict__ out) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t n = (int64_t)(P + NBC) * P;
+  if (i >= n) return;
+  const int64_t row = i / P, col = i % P;
+  out[i] = row < P ? Wd[i] : (row < P + NS ? WB[(row - P) * P + col] : WC[(row - P - NS) * P + col]);
+}
+
+__global__ void cvt_dbc_kernel(int64_t rows, int ldg, int P, const float* __restrict__ dbc, __nv_bfloat16* __restrict__ gcat) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= rows * NBC) return;
+  const int64_t row = i / NBC;
+  const int c = (int)(i % NBC);
+  gcat[row * ldg + P + c] = __float2bfloat16_rn(dbc[i]);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 row-major [rows, cols] with row pitch `ld` elements; box = {64 cols, box_rows}; 128-byte swizzle; OOB reads 0
+int make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return 1;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {ld * 2};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? 0 : 1;
+}
+
+template <int AMAJ, int BMAJ, int EPI>
+int launch_tc(const CUtensorMap& tmA, const CUtensorMap& tmB, const TcArgs& a, cudaStream_t st) {
+  static bool attr_set = false;
+  auto kern = gemm_tc_kernel<AMAJ, BMAJ, EPI>;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN) != cudaSuccess) return 1;
+    attr_set = true;
+  }
+  dim3 grid((unsigned)((a.M + BM - 1) / BM), (unsigned)((a.N + BN - 1) / BN), (unsigned)a.splitk);
+  kern<<<grid, 128, SMEM_DYN, st>>>(tmA, tmB, a);
+  count_launch();
+  return (int)cudaGetLastError();
+}
+
+}  // namespace
+
+int tc_pack_wcat(const Plan& pl, const as_params_t* pr, char* ws, cudaStream_t st) {
+  const int64_t n = (int64_t)(pl.P + NBC) * pl.P;
+  pack_wcat_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(
+      pl.P, (const __nv_bfloat16*)pr->W_delta, (const __nv_bfloat16*)pr->W_B, (const __nv_bfloat16*)pr->W_C,
+      (__nv_bfloat16*)(ws + pl.off_wcat));
+  count_launch();
+  return (int)cudaGetLastError();
+}
+
+int tc_projections(const Plan& pl, const as_params_t* pr, const void* x, char* ws, cudaStream_t st) {
+  const int64_t M = (int64_t)pl.B * pl.T;
+  const int P = pl.P, NW = P + NBC;
+  CUtensorMap tmA, tmB;
+  if (make_map(&tmA, x, M, P, P, BM)) return 1;
+  if (make_map(&tmB, ws + pl.off_wcat, NW, P, P, BN)) return 1;
+  TcArgs a{};
+  a.M = M; a.N = NW; a.kblocks = (P + BK - 1) / BK; a.splitk = 1; a.P = P;
+  a.delta = (float*)(ws + pl.off_delta); a.bc = (float*)(ws + pl.off_bc); a.bias = pr->b_delta;
+  a.status = (int*)(ws + pl.off_status);
+  return launch_tc<MAJ_K, MAJ_K, TC_PROJ>(tmA, tmB, a, st);
+}
+
+int tc_weight_grads(const Plan& pl, const void* x, const as_grads_t* out, char* ws, cudaStream_t st) {
+  const int64_t M = (int64_t)pl.B * pl.T;
+  const int P = pl.P, NW = P + NBC;
+  cvt_dbc_kernel<<<(unsigned)((M * NBC + 255) / 256), 256, 0, st>>>(M, NW, P, (const float*)(ws + pl.off_dbc),
+                                                                    (__nv_bfloat16*)(ws + pl.off_du));
+  count_launch();
+  if (cudaGetLastError() != cudaSuccess) return 1;
+  CUtensorMap tmA, tmB;
+  if (make_map(&tmA, ws + pl.off_du, M, NW, NW, 64)) return 1;   // Gcat as [K=tokens, M=P+32]
+  if (make_map(&tmB, x, M, P, P, 64)) return 1;                  // X as [K=tokens, N=P]
+  TcArgs a{};
+  a.M = NW; a.N = P; a.kblocks = (int)((M + BK - 1) / BK); a.P = P;
+  const int tiles = ((NW + BM - 1) / BM) * ((P + BN - 1) / BN);
+  int sk = (148 * 2 + tiles - 1) / tiles;
+  if (sk > a.kblocks) sk = a.kblocks;
+  if (sk < 1) sk = 1;
+  a.splitk = sk;
+  a.dW_delta = out->dW_delta; a.dW_B = out->dW_B; a.dW_C = out->dW_C;
+  a.status = (int*)(ws + pl.off_status);
+  return launch_tc<MAJ_MN, MAJ_MN, TC_DW>(tmA, tmB, a, st);
+}
+
+int tc_input_grad(const Plan& pl, void* dx, char* ws, cudaStream_t st) {
+  const int64_t M = (int64_t)pl.B * pl.T;
+  const int P = pl.P, NW = P + NBC;
+  CUtensorMap tmA, tmB;
+  if (make_map(&tmA, ws + pl.off_du, M, NW, NW, BM)) return 1;       // Gcat as [M=tokens, K=P+32]
+  if (make_map(&tmB, ws + pl.off_wcat, NW, P, P, 64)) return 1;      // Wcat as [K=P+32, N=P]
+  TcArgs a{};
+  a.M = M; a.N = P; a.kblocks = (NW + BK - 1) / BK; a.splitk = 1; a.P = P;
+  a.dxdir = (const __nv_bfloat16*)(ws + pl.off_dxdir); a.dx = (__nv_bfloat16*)dx;
+  a.status = (int*)(ws + pl.off_status);
+  return launch_tc<MAJ_K, MAJ_MN, TC_DX>(tmA, tmB, a, st);
+}
+
+}  // namespace as

@@ -55,10 +55,12 @@ struct Plan {
   int m;            // tbar / L   (whole segments inside a window that starts on a segment boundary)
   int r;            // tbar % L   (tokens of the following partial segment)
   int io;           // as_dtype_t
+  int tc;           // 1: bf16 tensor-core contractions (bf16 I/O and d_model % 32 == 0), 0: FP32-pipe GEMMs
+  int du_ld;        // row pitch (elements) of the du buffer: P, or P+32 when it is the left part of Gcat = [du|dB|dC]
   // byte offsets into the workspace
   size_t off_status, off_delta, off_bc, off_ckpt, off_cs, off_hend, off_muloc, off_mupart, off_segd,
       off_partd, off_firstd, off_hstart, off_carry, off_swin, off_du, off_dxdir, off_dbc, off_dxacc,
-      off_bptt_ckpt, total_fwd, total_grad;
+      off_bptt_ckpt, off_wcat, total_fwd, total_grad;
 };
 
 int make_plan(const as_shape_t* sh, int64_t tbar, Plan* pl);
@@ -87,6 +89,12 @@ int launch_fixup(const Plan& pl, const ScanPtrs& sp, bool with_mu, cudaStream_t 
 int launch_forward_y(const Plan& pl, const ScanPtrs& sp, void* y, cudaStream_t st);
 int launch_adjoint_main(const Plan& pl, const ScanPtrs& sp, float* dA_log, float* db_delta, cudaStream_t st);
 int launch_finish_dx(const Plan& pl, const float* dxacc, const void* dxdir, void* dx, cudaStream_t st);
+
+// bf16 tensor-core path (as_gemm_tc.cu)
+int tc_pack_wcat(const Plan& pl, const as_params_t* pr, char* ws, cudaStream_t st);
+int tc_projections(const Plan& pl, const as_params_t* pr, const void* x, char* ws, cudaStream_t st);
+int tc_weight_grads(const Plan& pl, const void* x, const as_grads_t* out, char* ws, cudaStream_t st);
+int tc_input_grad(const Plan& pl, void* dx, char* ws, cudaStream_t st);
 
 int launch_bptt(const Plan& pl, const ScanPtrs& sp, float* dA_log, float* db_delta, cudaStream_t st);
 

@@ -15,6 +15,8 @@ static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 int make_plan(const as_shape_t* sh, int64_t tbar, Plan* pl) {
   Plan p{};
   p.B = sh->batch; p.P = sh->d_model; p.T = sh->seqlen; p.io = sh->io;
+  p.tc = (sh->io == AS_BF16 && sh->d_model % 32 == 0) ? 1 : 0;
+  p.du_ld = p.tc ? p.P + NBC : p.P;
   p.full = tbar >= p.T;
   p.tbar = p.full ? p.T : tbar;
   const int64_t tiles = (int64_t)((p.P + CH - 1) / CH) * p.B;
@@ -42,6 +44,7 @@ int make_plan(const as_shape_t* sh, int64_t tbar, Plan* pl) {
   p.off_hend = take(BSPN * 4);
   p.off_segd = take(BSP * 4);
   p.off_hstart = take(BSPN * 4);
+  p.off_wcat = take((size_t)(p.P + NBC) * p.P * 2);
   p.total_fwd = o;
   p.off_ckpt = take((size_t)p.B * p.NC * p.P * NS * 4);
   p.off_cs = take((size_t)p.B * p.NC * p.P * 4);
@@ -51,7 +54,7 @@ int make_plan(const as_shape_t* sh, int64_t tbar, Plan* pl) {
   p.off_firstd = take(BSP * 4);
   p.off_carry = take(BSPN * 4);
   p.off_swin = take(BSP * 8);
-  p.off_du = take(BTP * e);
+  p.off_du = take(BT * (size_t)p.du_ld * e);
   p.off_dxdir = take(BTP * e);
   p.off_dbc = take(BT * NBC * 4);
   p.off_dxacc = take(BTP * 4);
@@ -426,7 +429,7 @@ adjoint_main_kernel(Plan pl, const IO* __restrict__ x, const IO* __restrict__ dy
         const float duv = ddelta * sig;
         dbacc += duv;
         if (active) {
-          st_io<IO>(du + row * P + p, duv);
+          st_io<IO>(du + row * pl.du_ld + p, duv);
           st_io<IO>(dxdir + row * P + p, d * ssum);
         }
         // transposing warp reduction: afterwards lane l holds the warp total of v[l]
