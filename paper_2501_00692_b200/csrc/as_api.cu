@@ -214,7 +214,7 @@ int as_ssm_forward(const as_shape_t* shape, const as_params_t* params, const voi
   e = projections(pl, params, x, w, st);
   if (e) return e;
   ScanPtrs sp{x, nullptr, params->A_log, w};
-  AS_TRY(launch_prepass(pl, sp, false, false, st));
+  AS_TRY(launch_prepass(pl, sp, false, st));
   AS_TRY(launch_fixup(pl, sp, false, st));
   AS_TRY(launch_forward_y(pl, sp, y, st));
   return AS_OK;
@@ -237,7 +237,7 @@ int as_adjoint_grad(const as_shape_t* shape, const as_params_t* params, const vo
   if (e) return e;
   mark(1, st);
   ScanPtrs sp{x, dy, params->A_log, w};
-  AS_TRY(launch_prepass(pl, sp, true, true, st));
+  AS_TRY(launch_prepass(pl, sp, true, st));
   mark(2, st);
   AS_TRY(launch_fixup(pl, sp, true, st));
   mark(3, st);

@@ -18,6 +18,7 @@ inline void count_launch(int n = 1) { g_launches.fetch_add(n); }
 constexpr int NS = 16;        // d_state handled by the scan kernels
 constexpr int CK = 8;         // tokens per checkpoint chunk (h of one chunk lives in registers)
 constexpr int CH = 128;       // channels per CTA of the scan kernels
+constexpr int TILE_FLOATS = CH * NS;   // one (channel tile, all states) block of a per-segment / per-chunk array
 constexpr int NBC = 2 * NS;   // per-token row of [B_t | C_t] (and of [dB_t | dC_t])
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
@@ -42,8 +43,10 @@ __device__ __forceinline__ float ex2_approx(float x) {
 
 // ---- time segmentation and scratch layout ---------------------------------------------------
 // Time is cut into S segments of L tokens (L a multiple of CK); a CTA owns (segment, batch element,
-// CH channels).  Per-(segment, channel, state) arrays use the float4-friendly order [.., 4, P, 4]
-// (state n = 4*q + r lives at ((q*P + p)*4 + r)) so that a warp's accesses are contiguous.
+// CH channels).  Per-(segment, channel, state) and per-(chunk, channel, state) arrays are stored as
+// blocks of TILE_FLOATS floats per channel tile, in the order the owning thread keeps them in registers
+// (float4 q of thread tid at float offset (q*CH + tid)*4), so one bulk copy moves a CTA's block and
+// every thread's access is a contiguous 16 bytes.
 struct Plan {
   int B, P;
   int64_t T;
@@ -55,6 +58,8 @@ struct Plan {
   int m;            // tbar / L   (whole segments inside a window that starts on a segment boundary)
   int r;            // tbar % L   (tokens of the following partial segment)
   int io;           // as_dtype_t
+  int tiles;        // ceil(P / CH) channel tiles
+  int bw;           // channels per staged row: min(CH, P)
   int tc;           // 1: bf16 tensor-core contractions (bf16 I/O and d_model % 32 == 0), 0: FP32-pipe GEMMs
   int du_ld;        // row pitch (elements) of the du buffer: P, or P+32 when it is the left part of Gcat = [du|dB|dC]
   // byte offsets into the workspace
@@ -84,7 +89,7 @@ struct ScanPtrs {
   const float* A_log;
   char* ws;
 };
-int launch_prepass(const Plan& pl, const ScanPtrs& sp, bool with_mu, bool with_ckpt, cudaStream_t st);
+int launch_prepass(const Plan& pl, const ScanPtrs& sp, bool with_mu, cudaStream_t st);
 int launch_fixup(const Plan& pl, const ScanPtrs& sp, bool with_mu, cudaStream_t st);
 int launch_forward_y(const Plan& pl, const ScanPtrs& sp, void* y, cudaStream_t st);
 int launch_adjoint_main(const Plan& pl, const ScanPtrs& sp, float* dA_log, float* db_delta, cudaStream_t st);

@@ -1,8 +1,17 @@
-// Time-segmented scan kernels: forward state recurrence, summed adjoint cotangent (reverse
-// recurrence with exact window exit) and the per-token vector-Jacobian products.
+// Time-segmented scan kernels: forward state recurrence, summed adjoint cotangent (reverse recurrence
+// with exact window exit) and the per-token vector-Jacobian products.
 //
-// Thread mapping: one thread per channel p holding the 16 states of that channel in registers;
-// a CTA owns CH channels of one batch element over one time segment.  B_t, C_t are warp-uniform.
+// Work decomposition: a CTA owns CH = 128 channels of one batch element over one time segment of L
+// tokens and walks it in chunks of CK = 8 tokens.  Inside a CTA, thread `tid` owns TWO channels
+// (tile*128 + 2*(tid/2), +1) and EIGHT of their 16 states (n = 8*(tid%2) + j): sums over states finish
+// with one shuffle between the two lanes of a pair, sums over channels (dB_t, dC_t) need a 16-value
+// transposing reduction over the 16 lanes of equal parity instead of 32 values over 32 lanes.
+// Arithmetic on the two states (2m, 2m+1) of a channel is packed into f32x2 instructions, which halves
+// the issue slots the FP32 pipe needs and leaves room for MUFU.EX2, shuffles and shared-memory loads.
+// Inputs of a chunk (x, Delta, dy tiles by 2D TMA; B/C rows, the chunk checkpoint and its cumulative
+// Delta by 1D bulk copies) land in a 3-stage shared-memory ring guarded by mbarriers with bounded waits.
+#include <cuda.h>
+
 #include "as_internal.cuh"
 
 namespace as {
@@ -19,9 +28,11 @@ int make_plan(const as_shape_t* sh, int64_t tbar, Plan* pl) {
   p.du_ld = p.tc ? p.P + NBC : p.P;
   p.full = tbar >= p.T;
   p.tbar = p.full ? p.T : tbar;
-  const int64_t tiles = (int64_t)((p.P + CH - 1) / CH) * p.B;
+  p.tiles = (p.P + CH - 1) / CH;
+  p.bw = p.P < CH ? p.P : CH;
+  const int64_t ctas = (int64_t)p.tiles * p.B;
   const int64_t target = 148 * 2 * 4;
-  int64_t s_target = (target + tiles - 1) / tiles;
+  int64_t s_target = (target + ctas - 1) / ctas;
   int64_t L = (p.T + s_target - 1) / s_target;
   L = (L + CK - 1) / CK * CK;
   if (L < 64) L = 64;
@@ -34,30 +45,30 @@ int make_plan(const as_shape_t* sh, int64_t tbar, Plan* pl) {
   const size_t e = sh->io == AS_BF16 ? 2 : 4;
   const size_t BTP = (size_t)p.B * p.T * p.P;
   const size_t BT = (size_t)p.B * p.T;
-  const size_t BSPN = (size_t)p.B * p.S * p.P * NS;
+  const size_t BSB = (size_t)p.B * p.S * p.tiles * TILE_FLOATS;   // per-(segment, channel, state) arrays
   const size_t BSP = (size_t)p.B * p.S * p.P;
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
   p.off_status = take(256);
   p.off_delta = take(BTP * 4);
-  p.off_bc = take(BT * NBC * 4);
-  p.off_hend = take(BSPN * 4);
+  p.off_bc = take((BT + CK) * NBC * 4);   // CK spare rows: a chunk's 1D copy may run past the last token
+  p.off_hend = take(BSB * 4);
   p.off_segd = take(BSP * 4);
-  p.off_hstart = take(BSPN * 4);
+  p.off_hstart = take(BSB * 4);
   p.off_wcat = take((size_t)(p.P + NBC) * p.P * 2);
   p.total_fwd = o;
-  p.off_ckpt = take((size_t)p.B * p.NC * p.P * NS * 4);
+  p.off_ckpt = take((size_t)p.B * p.NC * p.tiles * TILE_FLOATS * 4);
   p.off_cs = take((size_t)p.B * p.NC * p.P * 4);
-  p.off_muloc = take(BSPN * 4);
-  p.off_mupart = take(BSPN * 4);
+  p.off_muloc = take(BSB * 4);
+  p.off_mupart = take(BSB * 4);
   p.off_partd = take(BSP * 4);
   p.off_firstd = take(BSP * 4);
-  p.off_carry = take(BSPN * 4);
+  p.off_carry = take(BSB * 4);
   p.off_swin = take(BSP * 8);
   p.off_du = take(BT * (size_t)p.du_ld * e);
   p.off_dxdir = take(BTP * e);
   p.off_dbc = take(BT * NBC * 4);
-  p.off_dxacc = take(BTP * 4);
+  p.off_dxacc = take(p.tc ? 256 : BTP * 4);
   p.off_bptt_ckpt = take((size_t)p.B * ((p.T + 63) / 64) * p.P * NS * 4);
   p.total_grad = o;
   *pl = p;
@@ -66,214 +77,419 @@ int make_plan(const as_shape_t* sh, int64_t tbar, Plan* pl) {
 
 namespace {
 
-// index of state group q (0..3) of channel p in a [.., 4, P, 4] array, in float4 units
-__device__ __forceinline__ int64_t q4(int64_t base_pn, int P, int q, int p) {
-  return base_pn / 4 + (int64_t)q * P + p;
+typedef unsigned long long u64;   // two packed fp32 values (lo = even state, hi = odd state)
+
+__device__ __forceinline__ u64 pk(float lo, float hi) {
+  u64 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void upk(u64 v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c) {
+  u64 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ u64 mul2(u64 a, u64 b) {
+  u64 d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ u64 ex2_2(u64 e) {
+  float lo, hi;
+  upk(e, lo, hi);
+  return pk(ex2_approx(lo), ex2_approx(hi));
+}
+__device__ __forceinline__ float hsum(u64 v) {
+  float lo, hi;
+  upk(v, lo, hi);
+  return lo + hi;
 }
 
-__device__ __forceinline__ void load16(const float* arr, int64_t base_pn, int P, int p, float (&v)[NS]) {
-  const float4* a4 = reinterpret_cast<const float4*>(arr);
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    float4 t = __ldg(a4 + q4(base_pn, P, q, p));
-    v[4 * q] = t.x; v[4 * q + 1] = t.y; v[4 * q + 2] = t.z; v[4 * q + 3] = t.w;
-  }
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
 }
-__device__ __forceinline__ void store16(float* arr, int64_t base_pn, int P, int p, const float (&v)[NS]) {
-  float4* a4 = reinterpret_cast<float4*>(arr);
-#pragma unroll
-  for (int q = 0; q < 4; ++q)
-    a4[q4(base_pn, P, q, p)] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+constexpr uint32_t WAIT_LIMIT = 1u << 22;
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  const uint32_t addr = smem_u32(bar);
+  for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ void tma_2d(void* dst, const CUtensorMap* tm, int c0, int64_t c1, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(dst)), "l"(tm), "r"(c0), "r"((int)c1), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void bulk_1d(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
-__device__ __forceinline__ void load_bc(const float* bc_row, float (&Bt)[NS], float (&Ct)[NS]) {
-  const float4* r4 = reinterpret_cast<const float4*>(bc_row);
+template <typename IO> struct IoSz { static constexpr int v = sizeof(IO); };
+
+// shared-memory stage of one chunk
+template <int ESZ, bool WITH_G, bool WITH_CKPT, bool WIN>
+struct Stage {
+  static constexpr int X = 0;
+  static constexpr int D = X + CK * CH * ESZ;
+  static constexpr int BC = D + CK * CH * 4;
+  static constexpr int G = BC + CK * NBC * 4;
+  static constexpr int CKP = G + (WITH_G ? CK * CH * ESZ : 0);
+  static constexpr int CS = CKP + (WITH_CKPT ? TILE_FLOATS * 4 : 0);
+  static constexpr int G2 = CS + (WITH_CKPT ? CH * 4 : 0);
+  static constexpr int D2 = G2 + (WIN ? CK * CH * ESZ : 0);
+  static constexpr int BC2 = D2 + (WIN ? CK * CH * 4 : 0);
+  static constexpr int BYTES = BC2 + (WIN ? CK * NBC * 4 : 0);
+};
+constexpr int NSTAGE = 3;
+
+template <typename IO> __device__ __forceinline__ float2 lds_pair(const uint8_t* tile, int bw, int j, int k);
+template <> __device__ __forceinline__ float2 lds_pair<float>(const uint8_t* tile, int bw, int j, int k) {
+  return *reinterpret_cast<const float2*>(tile + ((size_t)j * bw + 2 * k) * 4);
+}
+template <> __device__ __forceinline__ float2 lds_pair<__nv_bfloat16>(const uint8_t* tile, int bw, int j, int k) {
+  const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(tile + ((size_t)j * bw + 2 * k) * 2);
+  return __bfloat1622float2(v);
+}
+
+struct Who {          // what this thread owns
+  int tid, k, half;   // pair index, state half
+  int pa;             // first channel (second is pa + 1)
+  bool act;           // channels exist (P is even, so both or neither)
+};
+__device__ __forceinline__ Who who(int tile, int P) {
+  Who w;
+  w.tid = threadIdx.x; w.k = w.tid >> 1; w.half = w.tid & 1;
+  w.pa = tile * CH + 2 * w.k;
+  w.act = w.pa < P;
+  return w;
+}
+// A2[u] = -exp(A_log) * log2(e) for unit u = ch*4 + m  ->  states (8*half + 2m, +1) of channel pa + ch
+__device__ __forceinline__ void load_A2(const float* A_log, const Who& w, u64 (&A2)[8]) {
+#pragma unroll
+  for (int u = 0; u < 8; ++u) {
+    float2 v = make_float2(0.f, 0.f);
+    if (w.act) v = __ldg(reinterpret_cast<const float2*>(A_log + (int64_t)(w.pa + u / 4) * NS + 8 * w.half + 2 * (u % 4)));
+    A2[u] = pk(-__expf(v.x) * LOG2E, -__expf(v.y) * LOG2E);
+  }
+}
+// 16 values of this thread inside a 2048-float tile block: float4 q of thread tid at (q*128 + tid)
+__device__ __forceinline__ void load_block(const float* blk, int tid, u64 (&v)[8]) {
+  const ulonglong2* b2 = reinterpret_cast<const ulonglong2*>(blk);
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
-    float4 t = __ldg(r4 + q);
-    Bt[4 * q] = t.x; Bt[4 * q + 1] = t.y; Bt[4 * q + 2] = t.z; Bt[4 * q + 3] = t.w;
-    float4 c = __ldg(r4 + 4 + q);
-    Ct[4 * q] = c.x; Ct[4 * q + 1] = c.y; Ct[4 * q + 2] = c.z; Ct[4 * q + 3] = c.w;
+    const ulonglong2 t = b2[q * CH + tid];
+    v[2 * q] = t.x; v[2 * q + 1] = t.y;
   }
+}
+__device__ __forceinline__ void load_block_g(const float* blk, int tid, u64 (&v)[8]) {
+  const ulonglong2* b2 = reinterpret_cast<const ulonglong2*>(blk);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const ulonglong2 t = __ldg(b2 + q * CH + tid);
+    v[2 * q] = t.x; v[2 * q + 1] = t.y;
+  }
+}
+__device__ __forceinline__ void store_block(float* blk, int tid, const u64 (&v)[8]) {
+  ulonglong2* b2 = reinterpret_cast<ulonglong2*>(blk);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) b2[q * CH + tid] = make_ulonglong2(v[2 * q], v[2 * q + 1]);
+}
+
+// sigmoid(u) from Delta = softplus(u): 1 - exp(-Delta), without cancellation for small Delta
+__device__ __forceinline__ float sig_from_delta(float d) {
+  const float big = 1.f - ex2_approx(-d * LOG2E);
+  float s = fmaf(-d, 1.f / 7.f, 1.f);
+  s = fmaf(-d * (1.f / 6.f), s, 1.f);
+  s = fmaf(-d * (1.f / 5.f), s, 1.f);
+  s = fmaf(-d * (1.f / 4.f), s, 1.f);
+  s = fmaf(-d * (1.f / 3.f), s, 1.f);
+  s = fmaf(-d * (1.f / 2.f), s, 1.f);
+  return d < 0.125f ? d * s : big;
 }
 
 // ------------------------------------------------------------------------------------------------
-// pre-pass: ascending local scan of one segment from h = 0.
-//   writes: state at the start of every CK-token chunk (relative to a zero segment start) and the
-//   local exclusive cumulative Delta there; the segment's end state and Delta sum; and, for the
-//   reverse recurrence, the segment-local cotangent sum referenced to the segment's first token
-//   mu_loc = sum_t gC_t prod_{j=start+1..t} abar_j, plus its snapshot after the first r tokens.
+// ascending pass over one segment.
+//   PRE_FWD : local scan from h = 0; writes the segment's end state and Delta sum.
+//   PRE_ADJ : PRE_FWD + the state at every chunk start (relative to a zero segment start) and the local
+//             exclusive cumulative Delta there, + the segment-local cotangent sum referenced to the segment's
+//             first token, mu_loc = sum_t gC_t prod_{j=start+1..t} abar_j, and its snapshot after r tokens.
+//   PRE_Y   : scan from the true segment-start state, writes y_t = sum_n C_t[n] h_t[n].
 // ------------------------------------------------------------------------------------------------
-template <typename IO, bool WITH_MU, bool WITH_CKPT>
-__global__ void __launch_bounds__(CH) prepass_kernel(Plan pl, const IO* __restrict__ x, const IO* __restrict__ dy,
-                                                     const float* __restrict__ A_log, char* __restrict__ ws) {
-  const int p = blockIdx.x * CH + threadIdx.x;
-  const int s = blockIdx.y, b = blockIdx.z;
-  const int P = pl.P;
-  if (p >= P) return;
-  const float* delta = reinterpret_cast<const float*>(ws + pl.off_delta);
-  const float* bc = reinterpret_cast<const float*>(ws + pl.off_bc);
-  float* ckpt = reinterpret_cast<float*>(ws + pl.off_ckpt);
-  float* cs = reinterpret_cast<float*>(ws + pl.off_cs);
+enum { PRE_FWD = 0, PRE_ADJ = 1, PRE_Y = 2 };
 
-  float A2[NS], h[NS], Pr[NS], acc[NS], snap[NS];
-#pragma unroll
-  for (int n = 0; n < NS; ++n) {
-    A2[n] = -__expf(__ldg(A_log + (int64_t)p * NS + n)) * LOG2E;
-    h[n] = 0.f; Pr[n] = 1.f; acc[n] = 0.f; snap[n] = 0.f;
-  }
+template <typename IO, int MODE>
+__global__ void __launch_bounds__(CH) ascend_kernel(const __grid_constant__ CUtensorMap tmX,
+                                                    const __grid_constant__ CUtensorMap tmD,
+                                                    const __grid_constant__ CUtensorMap tmG, Plan pl,
+                                                    const float* __restrict__ A_log, char* __restrict__ ws,
+                                                    IO* __restrict__ y) {
+  constexpr int ESZ = IoSz<IO>::v;
+  constexpr bool MU = MODE == PRE_ADJ;
+  using St = Stage<ESZ, MU, false, false>;
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[NSTAGE];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
+
+  const int tile = blockIdx.x, s = blockIdx.y, b = blockIdx.z;
+  const int P = pl.P, bw = pl.bw;
+  const Who w = who(tile, P);
   const int64_t t0 = (int64_t)s * pl.L;
   const int64_t t1 = min(pl.T, t0 + pl.L);
-  float cum = 0.f, partd = 0.f, firstd = 0.f;
-  for (int64_t t = t0; t < t1; ++t) {
-    const int64_t row = (int64_t)b * pl.T + t;
-    if (WITH_CKPT && ((t - t0) % CK) == 0) {
-      const int64_t c = (int64_t)b * pl.NC + t / CK;
-      store16(ckpt, c * P * NS, P, p, h);
-      cs[c * P + p] = cum;
-    }
-    const float dv = __ldg(delta + row * P + p);
-    const float xv = ld_io<IO>(x + row * P + p);
-    float Bt[NS], Ct[NS];
-    load_bc(bc + row * NBC, Bt, Ct);
-    const float dx = dv * xv;
-    float gv = 0.f;
-    if (WITH_MU) gv = ld_io<IO>(dy + row * P + p);
+  const int nchunk = (int)((t1 - t0 + CK - 1) / CK);
+  const float* bc = reinterpret_cast<const float*>(ws + pl.off_bc);
+  int* status = reinterpret_cast<int*>(ws + pl.off_status);
+
+  if (w.tid == 0) {
+    for (int i = 0; i < NSTAGE; ++i) mbar_init(&full_bar[i], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const uint32_t tx_bytes = (uint32_t)(CK * bw * ESZ * (MU ? 2 : 1) + CK * bw * 4 + CK * NBC * 4);
+  auto issue = [&](int c) {   // thread 0: stage chunk c
+    const int st = c % NSTAGE;
+    uint8_t* sm = smem + st * St::BYTES;
+    const int64_t row = (int64_t)b * pl.T + t0 + (int64_t)c * CK;
+    mbar_expect_tx(&full_bar[st], tx_bytes);
+    tma_2d(sm + St::X, &tmX, tile * CH, row, &full_bar[st]);
+    tma_2d(sm + St::D, &tmD, tile * CH, row, &full_bar[st]);
+    if (MU) tma_2d(sm + St::G, &tmG, tile * CH, row, &full_bar[st]);
+    bulk_1d(sm + St::BC, bc + row * NBC, CK * NBC * 4, &full_bar[st]);
+  };
+  if (w.tid == 0)
+    for (int c = 0; c < NSTAGE && c < nchunk; ++c) issue(c);
+
+  u64 A2[8], h[8], Pr[8], acc[8], snap[8];
+  load_A2(A_log, w, A2);
+  const int64_t sb = ((int64_t)b * pl.S + s) * pl.tiles + tile;
+  if (MODE == PRE_Y) {
+    load_block_g(reinterpret_cast<const float*>(ws + pl.off_hstart) + sb * TILE_FLOATS, w.tid, h);
+  } else {
 #pragma unroll
-    for (int n = 0; n < NS; ++n) {
-      const float a = ex2_approx(dv * A2[n]);
-      h[n] = fmaf(a, h[n], dx * Bt[n]);
-      if (WITH_MU) {
-        if (t > t0) Pr[n] *= a;
-        acc[n] = fmaf(gv * Ct[n], Pr[n], acc[n]);
+    for (int u = 0; u < 8; ++u) h[u] = 0ull;
+  }
+#pragma unroll
+  for (int u = 0; u < 8; ++u) { Pr[u] = pk(1.f, 1.f); acc[u] = 0ull; snap[u] = 0ull; }
+  float cum[2] = {0.f, 0.f}, partd[2] = {0.f, 0.f}, firstd[2] = {0.f, 0.f};
+
+  for (int c = 0; c < nchunk; ++c) {
+    const int st = c % NSTAGE;
+    const uint8_t* sm = smem + st * St::BYTES;
+    const bool ok = mbar_wait(&full_bar[st], (c / NSTAGE) & 1);
+    const int64_t tc = t0 + (int64_t)c * CK;
+    const int nt = (int)min((int64_t)CK, t1 - tc);
+    if (MODE == PRE_ADJ) {
+      const int64_t cc = ((int64_t)b * pl.NC + tc / CK);
+      store_block(reinterpret_cast<float*>(ws + pl.off_ckpt) + (cc * pl.tiles + tile) * TILE_FLOATS, w.tid, h);
+      if (w.half == 0 && w.act)
+        *reinterpret_cast<float2*>(reinterpret_cast<float*>(ws + pl.off_cs) + cc * P + w.pa) = make_float2(cum[0], cum[1]);
+    }
+    if (ok) {
+#pragma unroll
+      for (int j = 0; j < CK; ++j) {
+        if (j < nt) {
+          float2 dv = make_float2(0.f, 0.f), xv = dv, gv = dv;
+          if (w.act) {
+            dv = lds_pair<float>(sm + St::D, bw, j, w.k);
+            xv = lds_pair<IO>(sm + St::X, bw, j, w.k);
+            if (MU) gv = lds_pair<IO>(sm + St::G, bw, j, w.k);
+          }
+          const float* brow = reinterpret_cast<const float*>(sm + St::BC) + j * NBC + 8 * w.half;
+          const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
+          const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
+          const u64 Bp[4] = {b01.x, b01.y, b23.x, b23.y};
+          u64 Cp[4] = {0ull, 0ull, 0ull, 0ull};
+          if (MODE != PRE_FWD) {
+            const ulonglong2 c01 = *reinterpret_cast<const ulonglong2*>(brow + NS);
+            const ulonglong2 c23 = *reinterpret_cast<const ulonglong2*>(brow + NS + 4);
+            Cp[0] = c01.x; Cp[1] = c01.y; Cp[2] = c23.x; Cp[3] = c23.y;
+          }
+          const float dd[2] = {dv.x, dv.y};
+          const float dxs[2] = {dv.x * xv.x, dv.y * xv.y};
+          const float gs[2] = {gv.x, gv.y};
+          const bool first = (c == 0 && j == 0);
+          float yv[2] = {0.f, 0.f};
+#pragma unroll
+          for (int ch = 0; ch < 2; ++ch) {
+            const u64 d2 = pk(dd[ch], dd[ch]), dx2 = pk(dxs[ch], dxs[ch]), g2 = pk(gs[ch], gs[ch]);
+            u64 yacc = 0ull;
+#pragma unroll
+            for (int m = 0; m < 4; ++m) {
+              const int u = ch * 4 + m;
+              const u64 a = ex2_2(mul2(d2, A2[u]));
+              h[u] = fma2(a, h[u], mul2(dx2, Bp[m]));
+              if (MU) {
+                if (!first) Pr[u] = mul2(Pr[u], a);
+                acc[u] = fma2(mul2(g2, Cp[m]), Pr[u], acc[u]);
+              }
+              if (MODE == PRE_Y) yacc = fma2(Cp[m], h[u], yacc);
+            }
+            if (MODE == PRE_Y) yv[ch] = hsum(yacc);
+            if (first) firstd[ch] = dd[ch];
+            cum[ch] += dd[ch];
+          }
+          if (MODE == PRE_Y) {
+            yv[0] += __shfl_xor_sync(0xffffffffu, yv[0], 1);
+            yv[1] += __shfl_xor_sync(0xffffffffu, yv[1], 1);
+            if (w.act) st_io<IO>(y + ((int64_t)b * pl.T + tc + j) * P + w.pa + w.half, w.half ? yv[1] : yv[0]);
+          }
+          if (MU && (tc + j - t0 + 1) == pl.r) {
+            partd[0] = cum[0]; partd[1] = cum[1];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) snap[u] = acc[u];
+          }
+        }
       }
     }
-    if (t == t0) firstd = dv;
-    cum += dv;
-    if (WITH_MU && (t - t0 + 1) == pl.r) {
-      partd = cum;
+    const int bad = __syncthreads_or(ok ? 0 : 1);
+    if (bad) {
+      if (w.tid == 0) atomicExch(status, AS_ERR_TIMEOUT);
+      return;
+    }
+    if (w.tid == 0 && c + NSTAGE < nchunk) issue(c + NSTAGE);
+  }
+  if (MODE == PRE_Y) return;
+  if (MU && (t1 - t0) < pl.r) {   // ragged last segment shorter than r tokens: the snapshot is the whole segment
+    partd[0] = cum[0]; partd[1] = cum[1];
 #pragma unroll
-      for (int n = 0; n < NS; ++n) snap[n] = acc[n];
+    for (int u = 0; u < 8; ++u) snap[u] = acc[u];
+  }
+  store_block(reinterpret_cast<float*>(ws + pl.off_hend) + sb * TILE_FLOATS, w.tid, h);
+  const int64_t sp = ((int64_t)b * pl.S + s) * P + w.pa;
+  if (w.half == 0 && w.act) {
+    *reinterpret_cast<float2*>(reinterpret_cast<float*>(ws + pl.off_segd) + sp) = make_float2(cum[0], cum[1]);
+    if (MU) {
+      *reinterpret_cast<float2*>(reinterpret_cast<float*>(ws + pl.off_partd) + sp) = make_float2(partd[0], partd[1]);
+      *reinterpret_cast<float2*>(reinterpret_cast<float*>(ws + pl.off_firstd) + sp) = make_float2(firstd[0], firstd[1]);
     }
   }
-  if (WITH_MU && (t1 - t0) < pl.r) {   // ragged last segment shorter than r tokens: the snapshot is the whole segment
-    partd = cum;
-#pragma unroll
-    for (int n = 0; n < NS; ++n) snap[n] = acc[n];
-  }
-  const int64_t sb = (int64_t)b * pl.S + s;
-  store16(reinterpret_cast<float*>(ws + pl.off_hend), sb * P * NS, P, p, h);
-  reinterpret_cast<float*>(ws + pl.off_segd)[sb * P + p] = cum;
-  if (WITH_MU) {
-    store16(reinterpret_cast<float*>(ws + pl.off_muloc), sb * P * NS, P, p, acc);
-    store16(reinterpret_cast<float*>(ws + pl.off_mupart), sb * P * NS, P, p, snap);
-    reinterpret_cast<float*>(ws + pl.off_partd)[sb * P + p] = partd;
-    reinterpret_cast<float*>(ws + pl.off_firstd)[sb * P + p] = firstd;
+  if (MU) {
+    store_block(reinterpret_cast<float*>(ws + pl.off_muloc) + sb * TILE_FLOATS, w.tid, acc);
+    store_block(reinterpret_cast<float*>(ws + pl.off_mupart) + sb * TILE_FLOATS, w.tid, snap);
   }
 }
 
 // ------------------------------------------------------------------------------------------------
-// carries across segments: one thread per (batch, channel, state).
-//   hstart[s]  true state entering segment s.
-//   carry[s]   abar_{e+1} * mu_{e+1} for e the last token of segment s, i.e. what the reverse
-//              recurrence inside segment s starts from (mu_{e+1} is the window sum that starts on
-//              the first token of segment s+1: m whole segments plus r tokens).
-//   swin[s]    sum of Delta over the Tbar tokens after e (fp64), for the window-exit factor.
+// carries across segments.  Thread (b, tile, tid) owns the same 16 (channel, state) slots as in the scans.
 // ------------------------------------------------------------------------------------------------
-__global__ void fixup_kernel(Plan pl, const float* __restrict__ A_log, char* __restrict__ ws, int with_mu) {
-  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const int P = pl.P, S = pl.S;
-  if (idx >= (int64_t)pl.B * P * NS) return;
-  const int n = (int)(idx % NS);
-  const int p = (int)((idx / NS) % P);
-  const int b = (int)(idx / ((int64_t)NS * P));
-  const float A2 = -__expf(__ldg(A_log + (int64_t)p * NS + n)) * LOG2E;
-  auto at = [&](int s) -> int64_t {  // float index of (b,s,p,n) in a [B,S,4,P,4] array
-    return (((int64_t)b * S + s) * 4 + n / 4) * (int64_t)P * 4 + (int64_t)p * 4 + (n % 4);
-  };
+// hstart[s]: true state entering segment s (sequential in s).
+__global__ void __launch_bounds__(CH) fixup_h_kernel(Plan pl, const float* __restrict__ A_log, char* __restrict__ ws) {
+  const int tile = blockIdx.x, b = blockIdx.y;
+  const Who w = who(tile, pl.P);
+  u64 A2[8], hs[8];
+  load_A2(A_log, w, A2);
+#pragma unroll
+  for (int u = 0; u < 8; ++u) hs[u] = 0ull;
   const float* hend = reinterpret_cast<const float*>(ws + pl.off_hend);
   const float* segd = reinterpret_cast<const float*>(ws + pl.off_segd);
   float* hstart = reinterpret_cast<float*>(ws + pl.off_hstart);
-  float hs = 0.f;
-  for (int s = 0; s < S; ++s) {
-    hstart[at(s)] = hs;
-    hs = fmaf(ex2_approx(A2 * segd[((int64_t)b * S + s) * P + p]), hs, hend[at(s)]);
+  constexpr int UN = 4;
+  for (int s0 = 0; s0 < pl.S; s0 += UN) {
+    u64 he[UN][8];
+    float2 sd[UN];
+#pragma unroll
+    for (int i = 0; i < UN; ++i) {
+      const int s = min(s0 + i, pl.S - 1);
+      const int64_t sb = ((int64_t)b * pl.S + s) * pl.tiles + tile;
+      load_block_g(hend + sb * TILE_FLOATS, w.tid, he[i]);
+      sd[i] = w.act ? __ldg(reinterpret_cast<const float2*>(segd + ((int64_t)b * pl.S + s) * pl.P + w.pa)) : make_float2(0.f, 0.f);
+    }
+#pragma unroll
+    for (int i = 0; i < UN; ++i) {
+      const int s = s0 + i;
+      if (s < pl.S) {
+        const int64_t sb = ((int64_t)b * pl.S + s) * pl.tiles + tile;
+        store_block(hstart + sb * TILE_FLOATS, w.tid, hs);
+        const u64 d2[2] = {pk(sd[i].x, sd[i].x), pk(sd[i].y, sd[i].y)};
+#pragma unroll
+        for (int u = 0; u < 8; ++u) hs[u] = fma2(ex2_2(mul2(d2[u / 4], A2[u])), hs[u], he[i][u]);
+      }
+    }
   }
-  if (!with_mu) return;
+}
+
+// carry[s] = abar_{e+1} * mu_{e+1} for e the last token of segment s: what the reverse recurrence inside
+// segment s starts from.  mu_{e+1} is the window sum that starts on the first token of segment s+1:
+// m whole segments plus the first r tokens of the next one (all later segments in the full form).
+// swin[s]: sum of Delta over the Tbar tokens after e (fp64), for the window-exit factor.
+__global__ void __launch_bounds__(CH) fixup_mu_kernel(Plan pl, const float* __restrict__ A_log, char* __restrict__ ws) {
+  const int tile = blockIdx.x, b = blockIdx.z;
+  const int P = pl.P, S = pl.S;
+  const Who w = who(tile, P);
+  u64 A2[8];
+  load_A2(A_log, w, A2);
   const float* muloc = reinterpret_cast<const float*>(ws + pl.off_muloc);
   const float* mupart = reinterpret_cast<const float*>(ws + pl.off_mupart);
+  const float* segd = reinterpret_cast<const float*>(ws + pl.off_segd);
   const float* partd = reinterpret_cast<const float*>(ws + pl.off_partd);
   const float* firstd = reinterpret_cast<const float*>(ws + pl.off_firstd);
   float* carry = reinterpret_cast<float*>(ws + pl.off_carry);
   double* swin = reinterpret_cast<double*>(ws + pl.off_swin);
-  auto sp = [&](int s) -> int64_t { return ((int64_t)b * S + s) * P + p; };
-  // decay over (start(s), start(s+1)]
-  auto dsh = [&](int s) -> float {
-    const float nxt = (s + 1 < S) ? firstd[sp(s + 1)] : 0.f;
-    return ex2_approx(A2 * (segd[sp(s)] - firstd[sp(s)] + nxt));
+  auto blk = [&](int s) -> int64_t { return (((int64_t)b * S + s) * pl.tiles + tile) * TILE_FLOATS; };
+  auto ld2 = [&](const float* arr, int s) -> float2 {
+    return (w.act && s < S) ? __ldg(reinterpret_cast<const float2*>(arr + ((int64_t)b * S + s) * P + w.pa)) : make_float2(0.f, 0.f);
+  };
+  // decay over (start(s), start(s+1)] applied to val, then + muloc[s]
+  auto step = [&](int sg, u64 (&val)[8]) {
+    const float2 sd = ld2(segd, sg), fd = ld2(firstd, sg), fn = ld2(firstd, sg + 1);
+    const float e0 = sd.x - fd.x + fn.x, e1 = sd.y - fd.y + fn.y;
+    const u64 d2[2] = {pk(e0, e0), pk(e1, e1)};
+    u64 ml[8];
+    load_block_g(muloc + blk(sg), w.tid, ml);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) val[u] = fma2(ex2_2(mul2(d2[u / 4], A2[u])), val[u], ml[u]);
+  };
+  auto finish = [&](int s, u64 (&val)[8]) {   // multiply by abar of the first token of segment s+1 and store
+    const float2 fn = ld2(firstd, s + 1);
+    const u64 d2[2] = {pk(fn.x, fn.x), pk(fn.y, fn.y)};
+    u64 out[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) out[u] = (s + 1 < S) ? mul2(val[u], ex2_2(mul2(d2[u / 4], A2[u]))) : 0ull;
+    store_block(carry + blk(s), w.tid, out);
   };
   if (pl.full) {
-    float mstart = 0.f;  // mu at the first token of segment s+1
+    if (blockIdx.y != 0) return;
+    u64 mstart[8];   // mu at the first token of segment s+1
+#pragma unroll
+    for (int u = 0; u < 8; ++u) mstart[u] = 0ull;
     for (int s = S - 1; s >= 0; --s) {
-      carry[at(s)] = (s + 1 < S) ? ex2_approx(A2 * firstd[sp(s + 1)]) * mstart : 0.f;
-      mstart = fmaf(dsh(s), mstart, muloc[at(s)]);
+      finish(s, mstart);
+      step(s, mstart);
     }
   } else {
-    for (int s = 0; s < S; ++s) {
-      const int s1 = s + 1;
-      float val = 0.f;
-      if (s1 < S) {
-        const int sp_ = s1 + pl.m;  // partial segment
-        val = (sp_ < S) ? mupart[at(sp_)] : 0.f;
-        for (int k = pl.m - 1; k >= 0; --k) {
-          const int sg = s1 + k;
-          val = (sg < S) ? fmaf(dsh(sg), val, muloc[at(sg)]) : 0.f;
-        }
-        val *= ex2_approx(A2 * firstd[sp(s1)]);
-      }
-      carry[at(s)] = val;
-      if (n == 0) {
-        double sw = 0.0;
-        for (int k = 1; k <= pl.m; ++k)
-          if (s + k < S) sw += (double)segd[sp(s + k)];
-        if (s + pl.m + 1 < S) sw += (double)partd[sp(s + pl.m + 1)];
-        swin[sp(s)] = sw;
-      }
-    }
-  }
-}
-
-// ------------------------------------------------------------------------------------------------
-// forward output pass: h from the true segment start, y_t = sum_n C_t[n] h_t[n].
-// ------------------------------------------------------------------------------------------------
-template <typename IO>
-__global__ void __launch_bounds__(CH) forward_y_kernel(Plan pl, const IO* __restrict__ x, const float* __restrict__ A_log,
-                                                       const char* __restrict__ ws, IO* __restrict__ y) {
-  const int p = blockIdx.x * CH + threadIdx.x;
-  const int s = blockIdx.y, b = blockIdx.z;
-  const int P = pl.P;
-  if (p >= P) return;
-  const float* delta = reinterpret_cast<const float*>(ws + pl.off_delta);
-  const float* bc = reinterpret_cast<const float*>(ws + pl.off_bc);
-  float A2[NS], h[NS];
+    const int s = blockIdx.y;
+    const int s1 = s + 1;
+    u64 val[8];
 #pragma unroll
-  for (int n = 0; n < NS; ++n) A2[n] = -__expf(__ldg(A_log + (int64_t)p * NS + n)) * LOG2E;
-  load16(reinterpret_cast<const float*>(ws + pl.off_hstart), ((int64_t)b * pl.S + s) * P * NS, P, p, h);
-  const int64_t t0 = (int64_t)s * pl.L;
-  const int64_t t1 = min(pl.T, t0 + pl.L);
-  for (int64_t t = t0; t < t1; ++t) {
-    const int64_t row = (int64_t)b * pl.T + t;
-    const float dv = __ldg(delta + row * P + p);
-    const float dx = dv * ld_io<IO>(x + row * P + p);
-    float Bt[NS], Ct[NS];
-    load_bc(bc + row * NBC, Bt, Ct);
-    float yv = 0.f;
-#pragma unroll
-    for (int n = 0; n < NS; ++n) {
-      h[n] = fmaf(ex2_approx(dv * A2[n]), h[n], dx * Bt[n]);
-      yv = fmaf(Ct[n], h[n], yv);
+    for (int u = 0; u < 8; ++u) val[u] = 0ull;
+    if (s1 + pl.m < S) load_block_g(mupart + blk(s1 + pl.m), w.tid, val);
+    for (int k = pl.m - 1; k >= 0; --k) {
+      const int sg = s1 + k;
+      if (sg < S) step(sg, val);
     }
-    st_io<IO>(y + row * P + p, yv);
+    finish(s, val);
+    if (w.half == 0 && w.act) {
+      double sw0 = 0.0, sw1 = 0.0;
+      for (int k = 1; k <= pl.m; ++k) { const float2 v = ld2(segd, s + k); sw0 += (double)v.x; sw1 += (double)v.y; }
+      const float2 pv = ld2(partd, s + pl.m + 1);
+      sw0 += (double)pv.x; sw1 += (double)pv.y;
+      double* dst = swin + ((int64_t)b * S + s) * P + w.pa;
+      dst[0] = sw0; dst[1] = sw1;
+    }
   }
 }
 
@@ -284,183 +500,273 @@ __global__ void __launch_bounds__(CH) forward_y_kernel(Plan pl, const IO* __rest
 // ------------------------------------------------------------------------------------------------
 template <typename IO, bool FULL>
 __global__ void __launch_bounds__(CH, 2)
-adjoint_main_kernel(Plan pl, const IO* __restrict__ x, const IO* __restrict__ dy, const float* __restrict__ A_log,
+adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmD,
+                    const __grid_constant__ CUtensorMap tmG, Plan pl, const float* __restrict__ A_log,
                     char* __restrict__ ws, float* __restrict__ dA_log, float* __restrict__ db_delta) {
-  __shared__ float red[CH / 32][CK][NBC];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int pp = blockIdx.x * CH + tid;
-  const int s = blockIdx.y, b = blockIdx.z;
-  const int P = pl.P;
-  const bool active = pp < P;
-  const int p = active ? pp : P - 1;   // inactive threads shadow a valid channel and contribute zeros
+  constexpr int ESZ = IoSz<IO>::v;
+  constexpr bool WIN = !FULL;
+  using St = Stage<ESZ, true, true, WIN>;
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[NSTAGE];
+  __shared__ float red[2][CH / 32][CK][NBC];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
 
-  const float* delta = reinterpret_cast<const float*>(ws + pl.off_delta);
+  const int tile = blockIdx.x, s = blockIdx.y, b = blockIdx.z;
+  const int P = pl.P, bw = pl.bw;
+  const Who w = who(tile, P);
+  const int lane = w.tid & 31, warp = w.tid >> 5;
+  const int64_t t0 = (int64_t)s * pl.L;
+  const int64_t t1 = min(pl.T, t0 + pl.L);
+  const int nchunk = (int)((t1 - t0 + CK - 1) / CK);
   const float* bc = reinterpret_cast<const float*>(ws + pl.off_bc);
   const float* ckpt = reinterpret_cast<const float*>(ws + pl.off_ckpt);
   const float* cs = reinterpret_cast<const float*>(ws + pl.off_cs);
   IO* du = reinterpret_cast<IO*>(ws + pl.off_du);
   IO* dxdir = reinterpret_cast<IO*>(ws + pl.off_dxdir);
   float* dbc = reinterpret_cast<float*>(ws + pl.off_dbc);
+  int* status = reinterpret_cast<int*>(ws + pl.off_status);
+  const int ncs = min(CH, P - tile * CH);   // channels of this tile that exist
+  const int64_t BT = (int64_t)pl.B * pl.T;
 
-  float A2[NS], mu[NS], dAacc[NS];
-  const int64_t sb = (int64_t)b * pl.S + s;
-#pragma unroll
-  for (int n = 0; n < NS; ++n) {
-    A2[n] = -__expf(__ldg(A_log + (int64_t)p * NS + n)) * LOG2E;
-    dAacc[n] = 0.f;
+  if (w.tid == 0) {
+    for (int i = 0; i < NSTAGE; ++i) mbar_init(&full_bar[i], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  load16(reinterpret_cast<const float*>(ws + pl.off_carry), sb * P * NS, P, p, mu);
-  if (!active) {
+  __syncthreads();
+  const uint32_t tx_base = (uint32_t)(CK * bw * ESZ * 2 + CK * bw * 4 + CK * NBC * 4 + TILE_FLOATS * 4 + ncs * 4 +
+                                      (WIN ? CK * bw * ESZ + CK * bw * 4 : 0));
+  // chunks are visited last to first: the i-th visited chunk is c = nchunk-1-i
+  auto issue = [&](int i) {
+    const int st = i % NSTAGE;
+    const int c = nchunk - 1 - i;
+    uint8_t* sm = smem + st * St::BYTES;
+    const int64_t tc = t0 + (int64_t)c * CK;
+    const int64_t row = (int64_t)b * pl.T + tc;
+    const int64_t cc = (int64_t)b * pl.NC + tc / CK;
+    const int64_t row2 = row + pl.tbar;          // first token leaving the window of this chunk's tokens
+    const bool win_rows = WIN && row2 < BT;      // its B/C rows exist (else no token of the chunk has t + Tbar < T)
+    mbar_expect_tx(&full_bar[st], tx_base + (win_rows ? CK * NBC * 4 : 0));
+    tma_2d(sm + St::X, &tmX, tile * CH, row, &full_bar[st]);
+    tma_2d(sm + St::D, &tmD, tile * CH, row, &full_bar[st]);
+    tma_2d(sm + St::G, &tmG, tile * CH, row, &full_bar[st]);
+    bulk_1d(sm + St::BC, bc + row * NBC, CK * NBC * 4, &full_bar[st]);
+    bulk_1d(sm + St::CKP, ckpt + (cc * pl.tiles + tile) * TILE_FLOATS, TILE_FLOATS * 4, &full_bar[st]);
+    bulk_1d(sm + St::CS, cs + cc * P + tile * CH, ncs * 4, &full_bar[st]);
+    if (WIN) {
+      // rows of the tokens leaving the window; past the end of the whole tensor TMA fills zeros, and rows
+      // that belong to the next batch element are never used (guarded by t + Tbar < T)
+      tma_2d(sm + St::G2, &tmG, tile * CH, row2, &full_bar[st]);
+      tma_2d(sm + St::D2, &tmD, tile * CH, row2, &full_bar[st]);
+      if (win_rows) bulk_1d(sm + St::BC2, bc + row2 * NBC, CK * NBC * 4, &full_bar[st]);
+    }
+  };
+  if (w.tid == 0)
+    for (int i = 0; i < NSTAGE && i < nchunk; ++i) issue(i);
+
+  u64 A2[8], mu[8], dAacc[8];
+  load_A2(A_log, w, A2);
+  const int64_t sb = ((int64_t)b * pl.S + s) * pl.tiles + tile;
+  load_block_g(reinterpret_cast<const float*>(ws + pl.off_carry) + sb * TILE_FLOATS, w.tid, mu);
+  u64 hst[8];
+  load_block_g(reinterpret_cast<const float*>(ws + pl.off_hstart) + sb * TILE_FLOATS, w.tid, hst);
 #pragma unroll
-    for (int n = 0; n < NS; ++n) mu[n] = 0.f;
+  for (int u = 0; u < 8; ++u) dAacc[u] = 0ull;
+  // least negative exponent scale of each channel over all 16 states (for the window-term skip test)
+  float a2max[2];
+#pragma unroll
+  for (int ch = 0; ch < 2; ++ch) {
+    float mx = -3.0e38f;
+#pragma unroll
+    for (int m = 0; m < 4; ++m) { float lo, hi; upk(A2[ch * 4 + m], lo, hi); mx = fmaxf(mx, fmaxf(lo, hi)); }
+    a2max[ch] = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
   }
-  float A2max = A2[0];  // least negative exponent scale: the slowest-decaying state
-#pragma unroll
-  for (int n = 1; n < NS; ++n) A2max = fmaxf(A2max, A2[n]);
-  double sw = 0.0;
-  if (!FULL) sw = reinterpret_cast<const double*>(ws + pl.off_swin)[sb * P + p];
+  double sw[2] = {0.0, 0.0};
+  if (WIN && w.act) {
+    const double* swp = reinterpret_cast<const double*>(ws + pl.off_swin) + ((int64_t)b * pl.S + s) * P + w.pa;
+    sw[0] = swp[0]; sw[1] = swp[1];
+  }
   float dbacc = 0.f;
+  const int pmine = w.pa + w.half;   // the channel whose per-token outputs this lane finalises
 
-  const int64_t t0 = (int64_t)s * pl.L;
-  const int64_t t1 = min(pl.T, t0 + pl.L);
-  const int nchunk = (int)((t1 - t0 + CK - 1) / CK);
-
-  for (int c = nchunk - 1; c >= 0; --c) {
+  for (int i = 0; i < nchunk; ++i) {
+    const int st = i % NSTAGE;
+    const int c = nchunk - 1 - i;
+    const uint8_t* sm = smem + st * St::BYTES;
+    const bool ok = mbar_wait(&full_bar[st], (i / NSTAGE) & 1);
     const int64_t tc = t0 + (int64_t)c * CK;
     const int nt = (int)min((int64_t)CK, t1 - tc);
-    float xv[CK], dv[CK], gv[CK];
+    const int rb = i & 1;
+    if (ok) {
+      // state at the chunk start: local checkpoint + decayed true segment-start state
+      u64 h[8];
+      load_block(reinterpret_cast<const float*>(sm + St::CKP), w.tid, h);
+      {
+        float2 csv = make_float2(0.f, 0.f);
+        if (w.act) csv = *reinterpret_cast<const float2*>(sm + St::CS + 8 * w.k);
+        const u64 c2[2] = {pk(csv.x, csv.x), pk(csv.y, csv.y)};
 #pragma unroll
-    for (int j = 0; j < CK; ++j) {
-      const int64_t row = (int64_t)b * pl.T + tc + j;
-      const bool ok = j < nt;
-      dv[j] = ok ? __ldg(delta + row * P + p) : 0.f;
-      xv[j] = ok ? ld_io<IO>(x + row * P + p) : 0.f;
-      gv[j] = (ok && active) ? ld_io<IO>(dy + row * P + p) : 0.f;
-    }
-    // state at the chunk start: local checkpoint + decayed true segment-start state
-    float hs[CK][NS];
-    float h[NS];
-    {
-      const int64_t cc = (int64_t)b * pl.NC + tc / CK;
-      float hst[NS];
-      load16(reinterpret_cast<const float*>(ws + pl.off_hstart), sb * P * NS, P, p, hst);
-      load16(ckpt, cc * P * NS, P, p, h);
-      const float csum = __ldg(cs + cc * P + p);
-#pragma unroll
-      for (int n = 0; n < NS; ++n) h[n] = fmaf(ex2_approx(A2[n] * csum), hst[n], h[n]);
-    }
-    // forward rebuild
-#pragma unroll
-    for (int j = 0; j < CK; ++j) {
-      if (j < nt) {
-        const int64_t row = (int64_t)b * pl.T + tc + j;
-        const float4* r4 = reinterpret_cast<const float4*>(bc + row * NBC);
-        const float dxj = dv[j] * xv[j];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const float4 bt = __ldg(r4 + q);
-          const float bb[4] = {bt.x, bt.y, bt.z, bt.w};
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const int n = 4 * q + k;
-            h[n] = fmaf(ex2_approx(dv[j] * A2[n]), h[n], dxj * bb[k]);
-          }
-        }
+        for (int u = 0; u < 8; ++u) h[u] = fma2(ex2_2(mul2(c2[u / 4], A2[u])), hst[u], h[u]);
       }
+      // forward rebuild of the chunk
+      u64 hs[CK][8];
 #pragma unroll
-      for (int n = 0; n < NS; ++n) hs[j][n] = h[n];
-    }
-    // reverse walk
+      for (int j = 0; j < CK; ++j) {
+        if (j < nt) {
+          float2 dv = make_float2(0.f, 0.f), xv = dv;
+          if (w.act) {
+            dv = lds_pair<float>(sm + St::D, bw, j, w.k);
+            xv = lds_pair<IO>(sm + St::X, bw, j, w.k);
+          }
+          const float* brow = reinterpret_cast<const float*>(sm + St::BC) + j * NBC + 8 * w.half;
+          const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
+          const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
+          const u64 Bp[4] = {b01.x, b01.y, b23.x, b23.y};
+          const u64 d2[2] = {pk(dv.x, dv.x), pk(dv.y, dv.y)};
+          const u64 dx2[2] = {pk(dv.x * xv.x, dv.x * xv.x), pk(dv.y * xv.y, dv.y * xv.y)};
 #pragma unroll
-    for (int j = CK - 1; j >= 0; --j) {
-      if (j < nt) {
-        const int64_t t = tc + j;
-        const int64_t row = (int64_t)b * pl.T + t;
-        float Bt[NS], Ct[NS];
-        load_bc(bc + row * NBC, Bt, Ct);
-        const float g = gv[j], d = dv[j], xx = xv[j];
-        const float dxj = d * xx;
-        // mu_i += g_i C_i   (mu already carries abar_{i+1} mu_{i+1})
+          for (int u = 0; u < 8; ++u) h[u] = fma2(ex2_2(mul2(d2[u / 4], A2[u])), h[u], mul2(dx2[u / 4], Bp[u % 4]));
+        }
 #pragma unroll
-        for (int n = 0; n < NS; ++n) mu[n] = fmaf(g, Ct[n], mu[n]);
-        if (!FULL) {
-          const int64_t t2 = t + pl.tbar;
-          if (t2 < pl.T) {
-            // exact exit of token t2 from the window: subtract W_i gC_{t2}, W_i = exp(A * sum_{j=i+1..t2} Delta_j)
-            const int64_t row2 = (int64_t)b * pl.T + t2;
-            const float d2 = __ldg(delta + row2 * P + p);
-            const float swf = (float)sw;
-            if (__any_sync(0xffffffffu, swf * A2max > -126.f)) {
-              const float g2 = active ? ld_io<IO>(dy + row2 * P + p) : 0.f;
-              const float4* c4 = reinterpret_cast<const float4*>(bc + row2 * NBC) + 4;
+        for (int u = 0; u < 8; ++u) hs[j][u] = h[u];
+      }
+      // reverse walk
 #pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                const float4 ct = __ldg(c4 + q);
-                const float cc2[4] = {ct.x, ct.y, ct.z, ct.w};
+      for (int j = CK - 1; j >= 0; --j) {
+        if (j < nt) {
+          const int64_t t = tc + j;
+          float2 dv = make_float2(0.f, 0.f), xv = dv, gv = dv;
+          if (w.act) {
+            dv = lds_pair<float>(sm + St::D, bw, j, w.k);
+            xv = lds_pair<IO>(sm + St::X, bw, j, w.k);
+            gv = lds_pair<IO>(sm + St::G, bw, j, w.k);
+          }
+          const float* brow = reinterpret_cast<const float*>(sm + St::BC) + j * NBC + 8 * w.half;
+          const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
+          const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
+          const ulonglong2 c01 = *reinterpret_cast<const ulonglong2*>(brow + NS);
+          const ulonglong2 c23 = *reinterpret_cast<const ulonglong2*>(brow + NS + 4);
+          const u64 Bp[4] = {b01.x, b01.y, b23.x, b23.y};
+          const u64 Cp[4] = {c01.x, c01.y, c23.x, c23.y};
+          const float dd[2] = {dv.x, dv.y}, xs[2] = {xv.x, xv.y}, gs[2] = {gv.x, gv.y};
+          const float dxs[2] = {dv.x * xv.x, dv.y * xv.y};
+          // mu_i += g_i C_i   (mu already carries abar_{i+1} mu_{i+1})
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                  const int n = 4 * q + k;
-                  mu[n] = fmaf(-ex2_approx(swf * A2[n]), g2 * cc2[k], mu[n]);
+          for (int u = 0; u < 8; ++u) mu[u] = fma2(pk(gs[u / 4], gs[u / 4]), Cp[u % 4], mu[u]);
+          if (WIN) {
+            const int64_t t2 = t + pl.tbar;
+            if (t2 < pl.T) {
+              // exact exit of token t2 from the window: subtract W_i gC_{t2}, W_i = exp(A * sum_{j=i+1..t2} Delta_j)
+              float2 d2v = make_float2(0.f, 0.f), g2v = d2v;
+              if (w.act) {
+                d2v = lds_pair<float>(sm + St::D2, bw, j, w.k);
+                g2v = lds_pair<IO>(sm + St::G2, bw, j, w.k);
+              }
+              const float swf[2] = {(float)sw[0], (float)sw[1]};
+              const bool live = w.act && (swf[0] * a2max[0] > -126.f || swf[1] * a2max[1] > -126.f);
+              if (__any_sync(0xffffffffu, live)) {
+                const float* crow = reinterpret_cast<const float*>(sm + St::BC2) + j * NBC + NS + 8 * w.half;
+                const ulonglong2 e01 = *reinterpret_cast<const ulonglong2*>(crow);
+                const ulonglong2 e23 = *reinterpret_cast<const ulonglong2*>(crow + 4);
+                const u64 C2p[4] = {e01.x, e01.y, e23.x, e23.y};
+                const float g2s[2] = {-g2v.x, -g2v.y};
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                  const u64 W = ex2_2(mul2(pk(swf[u / 4], swf[u / 4]), A2[u]));
+                  mu[u] = fma2(W, mul2(pk(g2s[u / 4], g2s[u / 4]), C2p[u % 4]), mu[u]);
                 }
               }
+              sw[0] += (double)dd[0] - (double)d2v.x;   // window of token t-1: (t-1, t-1+Tbar]
+              sw[1] += (double)dd[1] - (double)d2v.y;
+            } else {
+              sw[0] += (double)dd[0];   // token t+Tbar does not exist: the (clipped) window sum only grows
+              sw[1] += (double)dd[1];
             }
-            sw += (double)d - (double)d2;   // window of token t-1: (t-1, t-1+Tbar]
-          } else {
-            // token t+Tbar does not exist: the (clipped) window sum only grows
-            sw += (double)d;
           }
-        }
-        float v[NBC];
-        float ssum = 0.f, dsum = 0.f;
+          u64 vB[4], vC[4];
+          float ssum[2], dsum[2];
 #pragma unroll
-        for (int n = 0; n < NS; ++n) {
-          const float hn = hs[j][n];
-          v[n] = mu[n] * dxj;                    // dB partial
-          v[NS + n] = g * hn;                    // dC partial
-          ssum = fmaf(mu[n], Bt[n], ssum);
-          const float hb = fmaf(-dxj, Bt[n], hn);  // abar_i h_{i-1}
-          const float q = mu[n] * hb;
-          dsum = fmaf(q, A2[n], dsum);
-          dAacc[n] = fmaf(q, d, dAacc[n]);
-          mu[n] *= ex2_approx(d * A2[n]);        // ready for token i-1
-        }
-        const float ddelta = fmaf(dsum, LN2, xx * ssum);
-        const float sig = -expm1f(-d);           // sigmoid(u) = 1 - exp(-softplus(u))
-        const float duv = ddelta * sig;
-        dbacc += duv;
-        if (active) {
-          st_io<IO>(du + row * pl.du_ld + p, duv);
-          st_io<IO>(dxdir + row * P + p, d * ssum);
-        }
-        // transposing warp reduction: afterwards lane l holds the warp total of v[l]
+          for (int ch = 0; ch < 2; ++ch) {
+            const u64 d2 = pk(dd[ch], dd[ch]), dx2 = pk(dxs[ch], dxs[ch]), ndx2 = pk(-dxs[ch], -dxs[ch]);
+            const u64 g2 = pk(gs[ch], gs[ch]);
+            u64 sacc = 0ull, dacc = 0ull;
 #pragma unroll
-        for (int off = 16, cnt = 16; off >= 1; off >>= 1, cnt >>= 1) {
-          const bool up = (lane & off) != 0;
-#pragma unroll
-          for (int k = 0; k < cnt; ++k) {
-            const float send = up ? v[k] : v[k + cnt];
-            const float keep = up ? v[k + cnt] : v[k];
-            v[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+            for (int m = 0; m < 4; ++m) {
+              const int u = ch * 4 + m;
+              const u64 hn = hs[j][u];
+              vB[m] = ch == 0 ? mul2(mu[u], dx2) : fma2(mu[u], dx2, vB[m]);   // dB partial (two channels)
+              vC[m] = ch == 0 ? mul2(g2, hn) : fma2(g2, hn, vC[m]);           // dC partial
+              sacc = fma2(mu[u], Bp[m], sacc);
+              const u64 hb = fma2(ndx2, Bp[m], hn);                            // abar_i h_{i-1}
+              const u64 q = mul2(mu[u], hb);
+              dacc = fma2(q, A2[u], dacc);
+              dAacc[u] = fma2(q, d2, dAacc[u]);
+              mu[u] = mul2(mu[u], ex2_2(mul2(d2, A2[u])));                     // ready for token i-1
+            }
+            ssum[ch] = hsum(sacc);
+            dsum[ch] = hsum(dacc);
           }
+#pragma unroll
+          for (int ch = 0; ch < 2; ++ch) {
+            ssum[ch] += __shfl_xor_sync(0xffffffffu, ssum[ch], 1);
+            dsum[ch] += __shfl_xor_sync(0xffffffffu, dsum[ch], 1);
+          }
+          {
+            const float d = w.half ? dd[1] : dd[0], xx = w.half ? xs[1] : xs[0];
+            const float sv = w.half ? ssum[1] : ssum[0], dsv = w.half ? dsum[1] : dsum[0];
+            const float ddelta = fmaf(dsv, LN2, xx * sv);
+            const float duv = ddelta * sig_from_delta(d);
+            dbacc += duv;
+            if (w.act) {
+              const int64_t row = (int64_t)b * pl.T + t;
+              st_io<IO>(du + row * pl.du_ld + pmine, duv);
+              st_io<IO>(dxdir + row * P + pmine, d * sv);
+            }
+          }
+          // transposing reduction over the 16 lanes of equal parity: afterwards this lane holds the warp total of
+          // value (lane >> 1): values 0..7 = dB[8*half + .], 8..15 = dC[8*half + .]
+          float v[16];
+#pragma unroll
+          for (int m = 0; m < 4; ++m) { upk(vB[m], v[2 * m], v[2 * m + 1]); upk(vC[m], v[8 + 2 * m], v[8 + 2 * m + 1]); }
+#pragma unroll
+          for (int off = 16, cnt = 8; cnt >= 1; off >>= 1, cnt >>= 1) {
+            const bool up = (lane & off) != 0;
+#pragma unroll
+            for (int k = 0; k < cnt; ++k) {
+              const float send = up ? v[k] : v[k + cnt];
+              const float keep = up ? v[k + cnt] : v[k];
+              v[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+            }
+          }
+          const int vi = lane >> 1;
+          red[rb][warp][j][(vi & 8) * 2 + 8 * w.half + (vi & 7)] = v[0];
         }
-        red[warp][j][lane] = v[0];
       }
     }
-    __syncthreads();
-    for (int e = tid; e < nt * NBC; e += CH) {
-      const int j = e / NBC, i = e % NBC;
+    const int bad = __syncthreads_or(ok ? 0 : 1);
+    if (bad) {
+      if (w.tid == 0) atomicExch(status, AS_ERR_TIMEOUT);
+      return;
+    }
+    if (w.tid == 0 && i + NSTAGE < nchunk) issue(i + NSTAGE);
+    for (int e = w.tid; e < nt * NBC; e += CH) {
+      const int j = e / NBC, q = e % NBC;
       float sum = 0.f;
 #pragma unroll
-      for (int w = 0; w < CH / 32; ++w) sum += red[w][j][i];
-      atomicAdd(dbc + ((int64_t)b * pl.T + tc + j) * NBC + i, sum);
+      for (int wq = 0; wq < CH / 32; ++wq) sum += red[rb][wq][j][q];
+      atomicAdd(dbc + ((int64_t)b * pl.T + tc + j) * NBC + q, sum);
     }
-    __syncthreads();
   }
-  if (active) {
+  if (w.act) {
 #pragma unroll
-    for (int n = 0; n < NS; ++n)
-      atomicAdd(dA_log + (int64_t)p * NS + n, dAacc[n] * (A2[n] * LN2));
-    atomicAdd(db_delta + p, dbacc);
+    for (int u = 0; u < 8; ++u) {
+      float alo, ahi, vlo, vhi;
+      upk(A2[u], alo, ahi);
+      upk(dAacc[u], vlo, vhi);
+      float* dst = dA_log + (int64_t)(w.pa + u / 4) * NS + 8 * w.half + 2 * (u % 4);
+      atomicAdd(dst, vlo * (alo * LN2));
+      atomicAdd(dst + 1, vhi * (ahi * LN2));
+    }
+    atomicAdd(db_delta + pmine, dbacc);
   }
 }
 
@@ -471,57 +777,109 @@ __global__ void finish_dx_kernel(int64_t n, const float* __restrict__ acc, const
   if (i < n) st_io<IO>(dx + i, acc[i] + ld_io<IO>(dxdir + i));
 }
 
+// ---- tensor maps for the [B*T, P] activation tiles (box = CK tokens x bw channels, no swizzle) --------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+int act_map(CUtensorMap* tm, const void* base, const Plan& pl, int elem_bytes, bool is_bf16) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return 1;
+  cuuint64_t dims[2] = {(cuuint64_t)pl.P, (cuuint64_t)pl.B * (cuuint64_t)pl.T};
+  cuuint64_t strides[1] = {(cuuint64_t)pl.P * elem_bytes};
+  cuuint32_t box[2] = {(cuuint32_t)pl.bw, (cuuint32_t)CK};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(tm, is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                   const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? 0 : 1;
+}
+struct Maps { CUtensorMap x, d, g; };
+int make_maps(const Plan& pl, const ScanPtrs& sp, Maps* m) {
+  const bool bf = pl.io == AS_BF16;
+  const int e = bf ? 2 : 4;
+  if (act_map(&m->x, sp.x, pl, e, bf)) return 1;
+  if (act_map(&m->d, sp.ws + pl.off_delta, pl, 4, false)) return 1;
+  if (act_map(&m->g, sp.dy ? sp.dy : sp.x, pl, e, bf)) return 1;
+  return 0;
+}
+
+template <typename K>
+int set_smem(K kern, int bytes) {
+  return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess ? 0 : 1;
+}
+
+template <typename IO, int MODE>
+int launch_ascend_t(const Plan& pl, const ScanPtrs& sp, void* y, cudaStream_t st) {
+  Maps m;
+  if (make_maps(pl, sp, &m)) return 1;
+  using St = Stage<sizeof(IO), MODE == PRE_ADJ, false, false>;
+  const int bytes = NSTAGE * St::BYTES + 128;
+  auto kern = ascend_kernel<IO, MODE>;
+  static bool once = false;
+  if (!once) { if (set_smem(kern, bytes)) return 1; once = true; }
+  kern<<<dim3(pl.tiles, pl.S, pl.B), CH, bytes, st>>>(m.x, m.d, m.g, pl, sp.A_log, sp.ws, (IO*)y);
+  count_launch();
+  return (int)cudaGetLastError();
+}
+
+template <typename IO, bool FULL>
+int launch_main_t(const Plan& pl, const ScanPtrs& sp, float* dA_log, float* db_delta, cudaStream_t st) {
+  Maps m;
+  if (make_maps(pl, sp, &m)) return 1;
+  using St = Stage<sizeof(IO), true, true, !FULL>;
+  const int bytes = NSTAGE * St::BYTES + 128;
+  auto kern = adjoint_main_kernel<IO, FULL>;
+  static bool once = false;
+  if (!once) { if (set_smem(kern, bytes)) return 1; once = true; }
+  kern<<<dim3(pl.tiles, pl.S, pl.B), CH, bytes, st>>>(m.x, m.d, m.g, pl, sp.A_log, sp.ws, dA_log, db_delta);
+  count_launch();
+  return (int)cudaGetLastError();
+}
+
 }  // namespace
 
 // ------------------------------------------------------------------------------------------------
 // launchers
 // ------------------------------------------------------------------------------------------------
-static dim3 seg_grid(const Plan& pl) { return dim3((pl.P + CH - 1) / CH, pl.S, pl.B); }
-
-int launch_prepass(const Plan& pl, const ScanPtrs& sp, bool with_mu, bool with_ckpt, cudaStream_t st) {
-  const dim3 g = seg_grid(pl);
-#define AS_PRE(IO, MU, CKP) \
-  prepass_kernel<IO, MU, CKP><<<g, CH, 0, st>>>(pl, (const IO*)sp.x, (const IO*)sp.dy, sp.A_log, sp.ws)
-  if (pl.io == AS_BF16) {
-    if (with_mu) AS_PRE(__nv_bfloat16, true, true);
-    else if (with_ckpt) AS_PRE(__nv_bfloat16, false, true);
-    else AS_PRE(__nv_bfloat16, false, false);
-  } else {
-    if (with_mu) AS_PRE(float, true, true);
-    else if (with_ckpt) AS_PRE(float, false, true);
-    else AS_PRE(float, false, false);
-  }
-#undef AS_PRE
-  count_launch();
-  return (int)cudaGetLastError();
+int launch_prepass(const Plan& pl, const ScanPtrs& sp, bool with_mu, cudaStream_t st) {
+  if (pl.io == AS_BF16)
+    return with_mu ? launch_ascend_t<__nv_bfloat16, PRE_ADJ>(pl, sp, nullptr, st)
+                   : launch_ascend_t<__nv_bfloat16, PRE_FWD>(pl, sp, nullptr, st);
+  return with_mu ? launch_ascend_t<float, PRE_ADJ>(pl, sp, nullptr, st) : launch_ascend_t<float, PRE_FWD>(pl, sp, nullptr, st);
 }
 
 int launch_fixup(const Plan& pl, const ScanPtrs& sp, bool with_mu, cudaStream_t st) {
-  const int64_t n = (int64_t)pl.B * pl.P * NS;
-  fixup_kernel<<<(unsigned)((n + 127) / 128), 128, 0, st>>>(pl, sp.A_log, sp.ws, with_mu ? 1 : 0);
+  fixup_h_kernel<<<dim3(pl.tiles, pl.B), CH, 0, st>>>(pl, sp.A_log, sp.ws);
   count_launch();
+  if (with_mu) {
+    fixup_mu_kernel<<<dim3(pl.tiles, pl.full ? 1 : pl.S, pl.B), CH, 0, st>>>(pl, sp.A_log, sp.ws);
+    count_launch();
+  }
   return (int)cudaGetLastError();
 }
 
 int launch_forward_y(const Plan& pl, const ScanPtrs& sp, void* y, cudaStream_t st) {
-  const dim3 g = seg_grid(pl);
-  if (pl.io == AS_BF16)
-    forward_y_kernel<__nv_bfloat16><<<g, CH, 0, st>>>(pl, (const __nv_bfloat16*)sp.x, sp.A_log, sp.ws, (__nv_bfloat16*)y);
-  else
-    forward_y_kernel<float><<<g, CH, 0, st>>>(pl, (const float*)sp.x, sp.A_log, sp.ws, (float*)y);
-  count_launch();
-  return (int)cudaGetLastError();
+  if (pl.io == AS_BF16) return launch_ascend_t<__nv_bfloat16, PRE_Y>(pl, sp, y, st);
+  return launch_ascend_t<float, PRE_Y>(pl, sp, y, st);
 }
 
 int launch_adjoint_main(const Plan& pl, const ScanPtrs& sp, float* dA_log, float* db_delta, cudaStream_t st) {
-  const dim3 g = seg_grid(pl);
-#define AS_MAIN(IO, F) \
-  adjoint_main_kernel<IO, F><<<g, CH, 0, st>>>(pl, (const IO*)sp.x, (const IO*)sp.dy, sp.A_log, sp.ws, dA_log, db_delta)
-  if (pl.io == AS_BF16) { if (pl.full) AS_MAIN(__nv_bfloat16, true); else AS_MAIN(__nv_bfloat16, false); }
-  else { if (pl.full) AS_MAIN(float, true); else AS_MAIN(float, false); }
-#undef AS_MAIN
-  count_launch();
-  return (int)cudaGetLastError();
+  if (pl.io == AS_BF16)
+    return pl.full ? launch_main_t<__nv_bfloat16, true>(pl, sp, dA_log, db_delta, st)
+                   : launch_main_t<__nv_bfloat16, false>(pl, sp, dA_log, db_delta, st);
+  return pl.full ? launch_main_t<float, true>(pl, sp, dA_log, db_delta, st)
+                 : launch_main_t<float, false>(pl, sp, dA_log, db_delta, st);
 }
 
 int launch_finish_dx(const Plan& pl, const float* dxacc, const void* dxdir, void* dx, cudaStream_t st) {
