@@ -157,12 +157,12 @@ struct Stage {
 };
 constexpr int NSTAGE = 3;
 
-template <typename IO> __device__ __forceinline__ float2 lds_pair(const uint8_t* tile, int bw, int j, int k);
-template <> __device__ __forceinline__ float2 lds_pair<float>(const uint8_t* tile, int bw, int j, int k) {
-  return *reinterpret_cast<const float2*>(tile + ((size_t)j * bw + 2 * k) * 4);
+template <typename IO> __device__ __forceinline__ float2 lds_pair(const uint8_t* tile, int j, int k);
+template <> __device__ __forceinline__ float2 lds_pair<float>(const uint8_t* tile, int j, int k) {
+  return *reinterpret_cast<const float2*>(tile + (j * CH + 2 * k) * 4);
 }
-template <> __device__ __forceinline__ float2 lds_pair<__nv_bfloat16>(const uint8_t* tile, int bw, int j, int k) {
-  const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(tile + ((size_t)j * bw + 2 * k) * 2);
+template <> __device__ __forceinline__ float2 lds_pair<__nv_bfloat16>(const uint8_t* tile, int j, int k) {
+  const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(tile + (j * CH + 2 * k) * 2);
   return __bfloat1622float2(v);
 }
 
@@ -243,10 +243,11 @@ __global__ void __launch_bounds__(CH) ascend_kernel(const __grid_constant__ CUte
   using St = Stage<ESZ, MU, false, false>;
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[NSTAGE];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
+  uint8_t* smem = smem_raw + ((128u - (smem_u32(smem_raw) & 127u)) & 127u);   // stays a shared-space pointer
 
   const int tile = blockIdx.x, s = blockIdx.y, b = blockIdx.z;
-  const int P = pl.P, bw = pl.bw;
+  const int P = pl.P;
+  constexpr int bw = CH;
   const Who w = who(tile, P);
   const int64_t t0 = (int64_t)s * pl.L;
   const int64_t t1 = min(pl.T, t0 + pl.L);
@@ -302,12 +303,11 @@ __global__ void __launch_bounds__(CH) ascend_kernel(const __grid_constant__ CUte
 #pragma unroll
       for (int j = 0; j < CK; ++j) {
         if (j < nt) {
-          float2 dv = make_float2(0.f, 0.f), xv = dv, gv = dv;
-          if (w.act) {
-            dv = lds_pair<float>(sm + St::D, bw, j, w.k);
-            xv = lds_pair<IO>(sm + St::X, bw, j, w.k);
-            if (MU) gv = lds_pair<IO>(sm + St::G, bw, j, w.k);
-          }
+          // channels past P read the zero fill of the TMA box: Delta = x = g = 0 keeps their slots at zero
+          const float2 dv = lds_pair<float>(sm + St::D, j, w.k);
+          const float2 xv = lds_pair<IO>(sm + St::X, j, w.k);
+          float2 gv = make_float2(0.f, 0.f);
+          if (MU) gv = lds_pair<IO>(sm + St::G, j, w.k);
           const float* brow = reinterpret_cast<const float*>(sm + St::BC) + j * NBC + 8 * w.half;
           const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
           const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
@@ -509,10 +509,12 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[NSTAGE];
   __shared__ float red[2][CH / 32][CK][NBC];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
+  __shared__ ulonglong2 hst_s[4][CH];
+  uint8_t* smem = smem_raw + ((128u - (smem_u32(smem_raw) & 127u)) & 127u);   // stays a shared-space pointer
 
   const int tile = blockIdx.x, s = blockIdx.y, b = blockIdx.z;
-  const int P = pl.P, bw = pl.bw;
+  const int P = pl.P;
+  constexpr int bw = CH;
   const Who w = who(tile, P);
   const int lane = w.tid & 31, warp = w.tid >> 5;
   const int64_t t0 = (int64_t)s * pl.L;
@@ -567,8 +569,12 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   load_A2(A_log, w, A2);
   const int64_t sb = ((int64_t)b * pl.S + s) * pl.tiles + tile;
   load_block_g(reinterpret_cast<const float*>(ws + pl.off_carry) + sb * TILE_FLOATS, w.tid, mu);
-  u64 hst[8];
-  load_block_g(reinterpret_cast<const float*>(ws + pl.off_hstart) + sb * TILE_FLOATS, w.tid, hst);
+  {   // true segment-start state: parked in shared memory, read back once per chunk
+    u64 hst[8];
+    load_block_g(reinterpret_cast<const float*>(ws + pl.off_hstart) + sb * TILE_FLOATS, w.tid, hst);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) hst_s[q][w.tid] = make_ulonglong2(hst[2 * q], hst[2 * q + 1]);
+  }
 #pragma unroll
   for (int u = 0; u < 8; ++u) dAacc[u] = 0ull;
   // least negative exponent scale of each channel over all 16 states (for the window-term skip test)
@@ -596,27 +602,30 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     const int64_t tc = t0 + (int64_t)c * CK;
     const int nt = (int)min((int64_t)CK, t1 - tc);
     const int rb = i & 1;
+    // window Delta sum: fp64 value at the chunk's last token + an fp32 running offset inside the chunk
+    float swc[2] = {(float)sw[0], (float)sw[1]}, swl[2] = {0.f, 0.f};
     if (ok) {
       // state at the chunk start: local checkpoint + decayed true segment-start state
       u64 h[8];
       load_block(reinterpret_cast<const float*>(sm + St::CKP), w.tid, h);
       {
-        float2 csv = make_float2(0.f, 0.f);
-        if (w.act) csv = *reinterpret_cast<const float2*>(sm + St::CS + 8 * w.k);
+        float2 csv = *reinterpret_cast<const float2*>(sm + St::CS + 8 * w.k);
+        if (!w.act) csv = make_float2(0.f, 0.f);   // the 1D copy only covers existing channels
         const u64 c2[2] = {pk(csv.x, csv.x), pk(csv.y, csv.y)};
 #pragma unroll
-        for (int u = 0; u < 8; ++u) h[u] = fma2(ex2_2(mul2(c2[u / 4], A2[u])), hst[u], h[u]);
+        for (int q = 0; q < 4; ++q) {
+          const ulonglong2 hq = hst_s[q][w.tid];
+          h[2 * q] = fma2(ex2_2(mul2(c2[q / 2], A2[2 * q])), hq.x, h[2 * q]);
+          h[2 * q + 1] = fma2(ex2_2(mul2(c2[q / 2], A2[2 * q + 1])), hq.y, h[2 * q + 1]);
+        }
       }
       // forward rebuild of the chunk
       u64 hs[CK][8];
 #pragma unroll
       for (int j = 0; j < CK; ++j) {
         if (j < nt) {
-          float2 dv = make_float2(0.f, 0.f), xv = dv;
-          if (w.act) {
-            dv = lds_pair<float>(sm + St::D, bw, j, w.k);
-            xv = lds_pair<IO>(sm + St::X, bw, j, w.k);
-          }
+          const float2 dv = lds_pair<float>(sm + St::D, j, w.k);
+          const float2 xv = lds_pair<IO>(sm + St::X, j, w.k);
           const float* brow = reinterpret_cast<const float*>(sm + St::BC) + j * NBC + 8 * w.half;
           const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
           const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
@@ -634,12 +643,9 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
       for (int j = CK - 1; j >= 0; --j) {
         if (j < nt) {
           const int64_t t = tc + j;
-          float2 dv = make_float2(0.f, 0.f), xv = dv, gv = dv;
-          if (w.act) {
-            dv = lds_pair<float>(sm + St::D, bw, j, w.k);
-            xv = lds_pair<IO>(sm + St::X, bw, j, w.k);
-            gv = lds_pair<IO>(sm + St::G, bw, j, w.k);
-          }
+          const float2 dv = lds_pair<float>(sm + St::D, j, w.k);
+          const float2 xv = lds_pair<IO>(sm + St::X, j, w.k);
+          const float2 gv = lds_pair<IO>(sm + St::G, j, w.k);
           const float* brow = reinterpret_cast<const float*>(sm + St::BC) + j * NBC + 8 * w.half;
           const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
           const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
@@ -656,13 +662,12 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
             const int64_t t2 = t + pl.tbar;
             if (t2 < pl.T) {
               // exact exit of token t2 from the window: subtract W_i gC_{t2}, W_i = exp(A * sum_{j=i+1..t2} Delta_j)
-              float2 d2v = make_float2(0.f, 0.f), g2v = d2v;
-              if (w.act) {
-                d2v = lds_pair<float>(sm + St::D2, bw, j, w.k);
-                g2v = lds_pair<IO>(sm + St::G2, bw, j, w.k);
-              }
-              const float swf[2] = {(float)sw[0], (float)sw[1]};
-              const bool live = w.act && (swf[0] * a2max[0] > -126.f || swf[1] * a2max[1] > -126.f);
+              const float2 d2v = lds_pair<float>(sm + St::D2, j, w.k);
+              const float2 g2v = lds_pair<IO>(sm + St::G2, j, w.k);
+              const float swf[2] = {swc[0] + swl[0], swc[1] + swl[1]};
+              // skip when every factor W = 2^(A2 * sum) of the warp is below 2^-64: the term is then far
+              // below one rounding unit of mu
+              const bool live = w.act && (swf[0] * a2max[0] > -64.f || swf[1] * a2max[1] > -64.f);
               if (__any_sync(0xffffffffu, live)) {
                 const float* crow = reinterpret_cast<const float*>(sm + St::BC2) + j * NBC + NS + 8 * w.half;
                 const ulonglong2 e01 = *reinterpret_cast<const ulonglong2*>(crow);
@@ -675,11 +680,11 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
                   mu[u] = fma2(W, mul2(pk(g2s[u / 4], g2s[u / 4]), C2p[u % 4]), mu[u]);
                 }
               }
-              sw[0] += (double)dd[0] - (double)d2v.x;   // window of token t-1: (t-1, t-1+Tbar]
-              sw[1] += (double)dd[1] - (double)d2v.y;
+              swl[0] += dd[0] - d2v.x;   // window of token t-1: (t-1, t-1+Tbar]
+              swl[1] += dd[1] - d2v.y;
             } else {
-              sw[0] += (double)dd[0];   // token t+Tbar does not exist: the (clipped) window sum only grows
-              sw[1] += (double)dd[1];
+              swl[0] += dd[0];           // token t+Tbar does not exist: the (clipped) window sum only grows
+              swl[1] += dd[1];
             }
           }
           u64 vB[4], vC[4];
@@ -742,6 +747,8 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         }
       }
     }
+    if (WIN) { sw[0] += (double)swl[0]; sw[1] += (double)swl[1]; }
+    (void)swc;
     const int bad = __syncthreads_or(ok ? 0 : 1);
     if (bad) {
       if (w.tid == 0) atomicExch(status, AS_ERR_TIMEOUT);
@@ -797,7 +804,7 @@ int act_map(CUtensorMap* tm, const void* base, const Plan& pl, int elem_bytes, b
   if (!enc) return 1;
   cuuint64_t dims[2] = {(cuuint64_t)pl.P, (cuuint64_t)pl.B * (cuuint64_t)pl.T};
   cuuint64_t strides[1] = {(cuuint64_t)pl.P * elem_bytes};
-  cuuint32_t box[2] = {(cuuint32_t)pl.bw, (cuuint32_t)CK};
+  cuuint32_t box[2] = {(cuuint32_t)CH, (cuuint32_t)CK};   // wider than P when P < CH: the rest is zero-filled
   cuuint32_t estr[2] = {1, 1};
   CUresult r = enc(tm, is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
                    const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
