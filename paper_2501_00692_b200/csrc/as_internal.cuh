@@ -64,7 +64,7 @@ struct Plan {
   int du_ld;        // row pitch (elements) of the du buffer: P, or P+32 when it is the left part of Gcat = [du|dB|dC]
   // byte offsets into the workspace
   size_t off_status, off_delta, off_bc, off_ckpt, off_cs, off_hend, off_muloc, off_mupart, off_segd,
-      off_partd, off_firstd, off_hstart, off_carry, off_swin, off_du, off_dxdir, off_dbc, off_dxacc,
+      off_partd, off_hstart, off_carry, off_swin, off_du, off_dxdir, off_dbc, off_dxacc,
       off_bptt_ckpt, off_wcat, total_fwd, total_grad;
 };
 

@@ -62,7 +62,6 @@ int make_plan(const as_shape_t* sh, int64_t tbar, Plan* pl) {
   p.off_muloc = take(BSB * 4);
   p.off_mupart = take(BSB * 4);
   p.off_partd = take(BSP * 4);
-  p.off_firstd = take(BSP * 4);
   p.off_carry = take(BSB * 4);
   p.off_swin = take(BSP * 8);
   p.off_du = take(BT * (size_t)p.du_ld * e);
@@ -155,7 +154,8 @@ struct Stage {
   static constexpr int BC2 = D2 + (WIN ? CK * CH * 4 : 0);
   static constexpr int BYTES = BC2 + (WIN ? CK * NBC * 4 : 0);
 };
-constexpr int NSTAGE = 3;
+constexpr int NSTAGE = 3;        // ascending kernels
+constexpr int NSTAGE_MAIN = 2;   // main adjoint kernel: a chunk takes thousands of cycles, one chunk of lookahead suffices
 
 template <typename IO> __device__ __forceinline__ float2 lds_pair(const uint8_t* tile, int j, int k);
 template <> __device__ __forceinline__ float2 lds_pair<float>(const uint8_t* tile, int j, int k) {
@@ -226,11 +226,20 @@ __device__ __forceinline__ float sig_from_delta(float d) {
 // ascending pass over one segment.
 //   PRE_FWD : local scan from h = 0; writes the segment's end state and Delta sum.
 //   PRE_ADJ : PRE_FWD + the state at every chunk start (relative to a zero segment start) and the local
-//             exclusive cumulative Delta there, + the segment-local cotangent sum referenced to the segment's
-//             first token, mu_loc = sum_t gC_t prod_{j=start+1..t} abar_j, and its snapshot after r tokens.
+//             exclusive cumulative Delta there, + the segment-local cotangent sum carried to the token before
+//             the segment, mu_loc = sum_t gC_t prod_{j=start..t} abar_j, and its snapshot after r tokens.
 //   PRE_Y   : scan from the true segment-start state, writes y_t = sum_n C_t[n] h_t[n].
+// Tokens past the end of the sequence inside the last chunk are neutralised by zeroing their staged
+// Delta, dy and B/C rows (Delta = 0 gives abar = 1 and a zero input term), so the token code has no branches.
 // ------------------------------------------------------------------------------------------------
 enum { PRE_FWD = 0, PRE_ADJ = 1, PRE_Y = 2 };
+
+// zero the staged rows [nt, CK) of a [CK x CH] tile (row_bytes per token) - all threads of the CTA
+__device__ __forceinline__ void zero_rows(uint8_t* tile, int row_bytes, int nt, int tid) {
+  uint4* p = reinterpret_cast<uint4*>(tile + nt * row_bytes);
+  const int n16 = (CK - nt) * row_bytes / 16;
+  for (int i = tid; i < n16; i += CH) p[i] = make_uint4(0u, 0u, 0u, 0u);
+}
 
 template <typename IO, int MODE>
 __global__ void __launch_bounds__(CH) ascend_kernel(const __grid_constant__ CUtensorMap tmX,
@@ -247,7 +256,6 @@ __global__ void __launch_bounds__(CH) ascend_kernel(const __grid_constant__ CUte
 
   const int tile = blockIdx.x, s = blockIdx.y, b = blockIdx.z;
   const int P = pl.P;
-  constexpr int bw = CH;
   const Who w = who(tile, P);
   const int64_t t0 = (int64_t)s * pl.L;
   const int64_t t1 = min(pl.T, t0 + pl.L);
@@ -260,7 +268,7 @@ __global__ void __launch_bounds__(CH) ascend_kernel(const __grid_constant__ CUte
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
-  const uint32_t tx_bytes = (uint32_t)(CK * bw * ESZ * (MU ? 2 : 1) + CK * bw * 4 + CK * NBC * 4);
+  const uint32_t tx_bytes = (uint32_t)(CK * CH * ESZ * (MU ? 2 : 1) + CK * CH * 4 + CK * NBC * 4);
   auto issue = [&](int c) {   // thread 0: stage chunk c
     const int st = c % NSTAGE;
     uint8_t* sm = smem + st * St::BYTES;
@@ -285,73 +293,78 @@ __global__ void __launch_bounds__(CH) ascend_kernel(const __grid_constant__ CUte
   }
 #pragma unroll
   for (int u = 0; u < 8; ++u) { Pr[u] = pk(1.f, 1.f); acc[u] = 0ull; snap[u] = 0ull; }
-  float cum[2] = {0.f, 0.f}, partd[2] = {0.f, 0.f}, firstd[2] = {0.f, 0.f};
+  float cum[2] = {0.f, 0.f}, partd[2] = {0.f, 0.f};
 
   for (int c = 0; c < nchunk; ++c) {
     const int st = c % NSTAGE;
-    const uint8_t* sm = smem + st * St::BYTES;
+    uint8_t* sm = smem + st * St::BYTES;
     const bool ok = mbar_wait(&full_bar[st], (c / NSTAGE) & 1);
     const int64_t tc = t0 + (int64_t)c * CK;
     const int nt = (int)min((int64_t)CK, t1 - tc);
+    const int jr = MU ? (int)(t0 + pl.r - 1 - tc) : -1;   // slot of the r-th token of the segment, if in this chunk
     if (MODE == PRE_ADJ) {
       const int64_t cc = ((int64_t)b * pl.NC + tc / CK);
       store_block(reinterpret_cast<float*>(ws + pl.off_ckpt) + (cc * pl.tiles + tile) * TILE_FLOATS, w.tid, h);
       if (w.half == 0 && w.act)
         *reinterpret_cast<float2*>(reinterpret_cast<float*>(ws + pl.off_cs) + cc * P + w.pa) = make_float2(cum[0], cum[1]);
     }
+    if (nt < CK) {   // only the last chunk of a sequence
+      if (ok) {
+        zero_rows(sm + St::D, CH * 4, nt, w.tid);
+        zero_rows(sm + St::BC, NBC * 4, nt, w.tid);
+        if (MU) zero_rows(sm + St::G, CH * ESZ, nt, w.tid);
+      }
+      __syncthreads();
+    }
     if (ok) {
 #pragma unroll
       for (int j = 0; j < CK; ++j) {
-        if (j < nt) {
-          // channels past P read the zero fill of the TMA box: Delta = x = g = 0 keeps their slots at zero
-          const float2 dv = lds_pair<float>(sm + St::D, j, w.k);
-          const float2 xv = lds_pair<IO>(sm + St::X, j, w.k);
-          float2 gv = make_float2(0.f, 0.f);
-          if (MU) gv = lds_pair<IO>(sm + St::G, j, w.k);
-          const float* brow = reinterpret_cast<const float*>(sm + St::BC) + j * NBC + 8 * w.half;
-          const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
-          const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
-          const u64 Bp[4] = {b01.x, b01.y, b23.x, b23.y};
-          u64 Cp[4] = {0ull, 0ull, 0ull, 0ull};
-          if (MODE != PRE_FWD) {
-            const ulonglong2 c01 = *reinterpret_cast<const ulonglong2*>(brow + NS);
-            const ulonglong2 c23 = *reinterpret_cast<const ulonglong2*>(brow + NS + 4);
-            Cp[0] = c01.x; Cp[1] = c01.y; Cp[2] = c23.x; Cp[3] = c23.y;
-          }
-          const float dd[2] = {dv.x, dv.y};
-          const float dxs[2] = {dv.x * xv.x, dv.y * xv.y};
-          const float gs[2] = {gv.x, gv.y};
-          const bool first = (c == 0 && j == 0);
-          float yv[2] = {0.f, 0.f};
+        // channels past P read the zero fill of the TMA box: Delta = x = g = 0 keeps their slots at zero
+        const float2 dv = lds_pair<float>(sm + St::D, j, w.k);
+        const float2 xv = lds_pair<IO>(sm + St::X, j, w.k);
+        float2 gv = make_float2(0.f, 0.f);
+        if (MU) gv = lds_pair<IO>(sm + St::G, j, w.k);
+        const float* brow = reinterpret_cast<const float*>(sm + St::BC) + j * NBC + 8 * w.half;
+        const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
+        const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
+        const u64 Bp[4] = {b01.x, b01.y, b23.x, b23.y};
+        u64 Cp[4] = {0ull, 0ull, 0ull, 0ull};
+        if (MODE != PRE_FWD) {
+          const ulonglong2 c01 = *reinterpret_cast<const ulonglong2*>(brow + NS);
+          const ulonglong2 c23 = *reinterpret_cast<const ulonglong2*>(brow + NS + 4);
+          Cp[0] = c01.x; Cp[1] = c01.y; Cp[2] = c23.x; Cp[3] = c23.y;
+        }
+        const float dd[2] = {dv.x, dv.y};
+        const float dxs[2] = {dv.x * xv.x, dv.y * xv.y};
+        const float gs[2] = {gv.x, gv.y};
+        float yv[2] = {0.f, 0.f};
 #pragma unroll
-          for (int ch = 0; ch < 2; ++ch) {
-            const u64 d2 = pk(dd[ch], dd[ch]), dx2 = pk(dxs[ch], dxs[ch]), g2 = pk(gs[ch], gs[ch]);
-            u64 yacc = 0ull;
+        for (int ch = 0; ch < 2; ++ch) {
+          const u64 d2 = pk(dd[ch], dd[ch]), dx2 = pk(dxs[ch], dxs[ch]), g2 = pk(gs[ch], gs[ch]);
+          u64 yacc = 0ull;
 #pragma unroll
-            for (int m = 0; m < 4; ++m) {
-              const int u = ch * 4 + m;
-              const u64 a = ex2_2(mul2(d2, A2[u]));
-              h[u] = fma2(a, h[u], mul2(dx2, Bp[m]));
-              if (MU) {
-                if (!first) Pr[u] = mul2(Pr[u], a);
-                acc[u] = fma2(mul2(g2, Cp[m]), Pr[u], acc[u]);
-              }
-              if (MODE == PRE_Y) yacc = fma2(Cp[m], h[u], yacc);
+          for (int m = 0; m < 4; ++m) {
+            const int u = ch * 4 + m;
+            const u64 a = ex2_2(mul2(d2, A2[u]));
+            h[u] = fma2(a, h[u], mul2(dx2, Bp[m]));
+            if (MU) {
+              Pr[u] = mul2(Pr[u], a);
+              acc[u] = fma2(mul2(g2, Cp[m]), Pr[u], acc[u]);
             }
-            if (MODE == PRE_Y) yv[ch] = hsum(yacc);
-            if (first) firstd[ch] = dd[ch];
-            cum[ch] += dd[ch];
+            if (MODE == PRE_Y) yacc = fma2(Cp[m], h[u], yacc);
           }
-          if (MODE == PRE_Y) {
-            yv[0] += __shfl_xor_sync(0xffffffffu, yv[0], 1);
-            yv[1] += __shfl_xor_sync(0xffffffffu, yv[1], 1);
-            if (w.act) st_io<IO>(y + ((int64_t)b * pl.T + tc + j) * P + w.pa + w.half, w.half ? yv[1] : yv[0]);
-          }
-          if (MU && (tc + j - t0 + 1) == pl.r) {
-            partd[0] = cum[0]; partd[1] = cum[1];
+          if (MODE == PRE_Y) yv[ch] = hsum(yacc);
+          cum[ch] += dd[ch];
+        }
+        if (MODE == PRE_Y) {
+          yv[0] += __shfl_xor_sync(0xffffffffu, yv[0], 1);
+          yv[1] += __shfl_xor_sync(0xffffffffu, yv[1], 1);
+          if (w.act && j < nt) st_io<IO>(y + ((int64_t)b * pl.T + tc + j) * P + w.pa + w.half, w.half ? yv[1] : yv[0]);
+        }
+        if (MU && j == jr) {
+          partd[0] = cum[0]; partd[1] = cum[1];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) snap[u] = acc[u];
-          }
+          for (int u = 0; u < 8; ++u) snap[u] = acc[u];
         }
       }
     }
@@ -372,10 +385,7 @@ __global__ void __launch_bounds__(CH) ascend_kernel(const __grid_constant__ CUte
   const int64_t sp = ((int64_t)b * pl.S + s) * P + w.pa;
   if (w.half == 0 && w.act) {
     *reinterpret_cast<float2*>(reinterpret_cast<float*>(ws + pl.off_segd) + sp) = make_float2(cum[0], cum[1]);
-    if (MU) {
-      *reinterpret_cast<float2*>(reinterpret_cast<float*>(ws + pl.off_partd) + sp) = make_float2(partd[0], partd[1]);
-      *reinterpret_cast<float2*>(reinterpret_cast<float*>(ws + pl.off_firstd) + sp) = make_float2(firstd[0], firstd[1]);
-    }
+    if (MU) *reinterpret_cast<float2*>(reinterpret_cast<float*>(ws + pl.off_partd) + sp) = make_float2(partd[0], partd[1]);
   }
   if (MU) {
     store_block(reinterpret_cast<float*>(ws + pl.off_muloc) + sb * TILE_FLOATS, w.tid, acc);
@@ -423,8 +433,9 @@ __global__ void __launch_bounds__(CH) fixup_h_kernel(Plan pl, const float* __res
 }
 
 // carry[s] = abar_{e+1} * mu_{e+1} for e the last token of segment s: what the reverse recurrence inside
-// segment s starts from.  mu_{e+1} is the window sum that starts on the first token of segment s+1:
-// m whole segments plus the first r tokens of the next one (all later segments in the full form).
+// segment s starts from.  With mu_loc[s'] already carried to the token before segment s', this is
+//   mu_loc[s+1] + D[s+1] (mu_loc[s+2] + ... + D[s+m] mu_part[s+m+1]),   D[s'] = exp(A * sum of Delta over s'),
+// i.e. m whole segments plus the first r tokens of the next one (all later segments in the full form).
 // swin[s]: sum of Delta over the Tbar tokens after e (fp64), for the window-exit factor.
 __global__ void __launch_bounds__(CH) fixup_mu_kernel(Plan pl, const float* __restrict__ A_log, char* __restrict__ ws) {
   const int tile = blockIdx.x, b = blockIdx.z;
@@ -436,39 +447,28 @@ __global__ void __launch_bounds__(CH) fixup_mu_kernel(Plan pl, const float* __re
   const float* mupart = reinterpret_cast<const float*>(ws + pl.off_mupart);
   const float* segd = reinterpret_cast<const float*>(ws + pl.off_segd);
   const float* partd = reinterpret_cast<const float*>(ws + pl.off_partd);
-  const float* firstd = reinterpret_cast<const float*>(ws + pl.off_firstd);
   float* carry = reinterpret_cast<float*>(ws + pl.off_carry);
   double* swin = reinterpret_cast<double*>(ws + pl.off_swin);
   auto blk = [&](int s) -> int64_t { return (((int64_t)b * S + s) * pl.tiles + tile) * TILE_FLOATS; };
   auto ld2 = [&](const float* arr, int s) -> float2 {
     return (w.act && s < S) ? __ldg(reinterpret_cast<const float2*>(arr + ((int64_t)b * S + s) * P + w.pa)) : make_float2(0.f, 0.f);
   };
-  // decay over (start(s), start(s+1)] applied to val, then + muloc[s]
-  auto step = [&](int sg, u64 (&val)[8]) {
-    const float2 sd = ld2(segd, sg), fd = ld2(firstd, sg), fn = ld2(firstd, sg + 1);
-    const float e0 = sd.x - fd.x + fn.x, e1 = sd.y - fd.y + fn.y;
-    const u64 d2[2] = {pk(e0, e0), pk(e1, e1)};
+  auto step = [&](int sg, u64 (&val)[8]) {   // val = mu_loc[sg] + D[sg] * val
+    const float2 sd = ld2(segd, sg);
+    const u64 d2[2] = {pk(sd.x, sd.x), pk(sd.y, sd.y)};
     u64 ml[8];
     load_block_g(muloc + blk(sg), w.tid, ml);
 #pragma unroll
     for (int u = 0; u < 8; ++u) val[u] = fma2(ex2_2(mul2(d2[u / 4], A2[u])), val[u], ml[u]);
   };
-  auto finish = [&](int s, u64 (&val)[8]) {   // multiply by abar of the first token of segment s+1 and store
-    const float2 fn = ld2(firstd, s + 1);
-    const u64 d2[2] = {pk(fn.x, fn.x), pk(fn.y, fn.y)};
-    u64 out[8];
-#pragma unroll
-    for (int u = 0; u < 8; ++u) out[u] = (s + 1 < S) ? mul2(val[u], ex2_2(mul2(d2[u / 4], A2[u]))) : 0ull;
-    store_block(carry + blk(s), w.tid, out);
-  };
   if (pl.full) {
     if (blockIdx.y != 0) return;
-    u64 mstart[8];   // mu at the first token of segment s+1
+    u64 val[8];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) mstart[u] = 0ull;
+    for (int u = 0; u < 8; ++u) val[u] = 0ull;
     for (int s = S - 1; s >= 0; --s) {
-      finish(s, mstart);
-      step(s, mstart);
+      store_block(carry + blk(s), w.tid, val);
+      step(s, val);
     }
   } else {
     const int s = blockIdx.y;
@@ -481,7 +481,7 @@ __global__ void __launch_bounds__(CH) fixup_mu_kernel(Plan pl, const float* __re
       const int sg = s1 + k;
       if (sg < S) step(sg, val);
     }
-    finish(s, val);
+    store_block(carry + blk(s), w.tid, val);
     if (w.half == 0 && w.act) {
       double sw0 = 0.0, sw1 = 0.0;
       for (int k = 1; k <= pl.m; ++k) { const float2 v = ld2(segd, s + k); sw0 += (double)v.x; sw1 += (double)v.y; }
@@ -495,11 +495,14 @@ __global__ void __launch_bounds__(CH) fixup_mu_kernel(Plan pl, const float* __re
 
 // ------------------------------------------------------------------------------------------------
 // main adjoint kernel: descending over the CK-token chunks of one segment.
-//   per chunk: rebuild h for the chunk from its checkpoint, then walk it backwards updating the summed
-//   cotangent mu_i = gC_i + abar_{i+1} mu_{i+1} - W_i gC_{i+Tbar} and evaluating the per-token VJPs.
+//   per chunk: rebuild h for the chunk from its checkpoint (keeping only every other token's state in
+//   registers; the odd tokens' states are rebuilt in the backward walk from the abar they need anyway),
+//   then walk it backwards updating the summed cotangent
+//       mu_i = gC_i + abar_{i+1} mu_{i+1} - W_i gC_{i+Tbar}
+//   and evaluating the per-token VJPs.
 // ------------------------------------------------------------------------------------------------
 template <typename IO, bool FULL>
-__global__ void __launch_bounds__(CH, 2)
+__global__ void __launch_bounds__(CH, 3)
 adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmD,
                     const __grid_constant__ CUtensorMap tmG, Plan pl, const float* __restrict__ A_log,
                     char* __restrict__ ws, float* __restrict__ dA_log, float* __restrict__ db_delta) {
@@ -507,45 +510,47 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   constexpr bool WIN = !FULL;
   using St = Stage<ESZ, true, true, WIN>;
   extern __shared__ __align__(128) uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t full_bar[NSTAGE];
+  __shared__ __align__(8) uint64_t full_bar[NSTAGE_MAIN];
   __shared__ float red[2][CH / 32][CK][NBC];
   __shared__ ulonglong2 hst_s[4][CH];
   uint8_t* smem = smem_raw + ((128u - (smem_u32(smem_raw) & 127u)) & 127u);   // stays a shared-space pointer
 
   const int tile = blockIdx.x, s = blockIdx.y, b = blockIdx.z;
   const int P = pl.P;
-  constexpr int bw = CH;
   const Who w = who(tile, P);
   const int lane = w.tid & 31, warp = w.tid >> 5;
+  const int64_t T = pl.T, tbar = pl.tbar;
   const int64_t t0 = (int64_t)s * pl.L;
-  const int64_t t1 = min(pl.T, t0 + pl.L);
+  const int64_t t1 = min(T, t0 + pl.L);
   const int nchunk = (int)((t1 - t0 + CK - 1) / CK);
   const float* bc = reinterpret_cast<const float*>(ws + pl.off_bc);
   const float* ckpt = reinterpret_cast<const float*>(ws + pl.off_ckpt);
   const float* cs = reinterpret_cast<const float*>(ws + pl.off_cs);
-  IO* du = reinterpret_cast<IO*>(ws + pl.off_du);
-  IO* dxdir = reinterpret_cast<IO*>(ws + pl.off_dxdir);
   float* dbc = reinterpret_cast<float*>(ws + pl.off_dbc);
   int* status = reinterpret_cast<int*>(ws + pl.off_status);
   const int ncs = min(CH, P - tile * CH);   // channels of this tile that exist
-  const int64_t BT = (int64_t)pl.B * pl.T;
+  const int64_t BT = (int64_t)pl.B * T;
+  const int du_ld = pl.du_ld;
+  const int pmine = w.pa + w.half;   // the channel whose per-token outputs this lane finalises
+  IO* du = reinterpret_cast<IO*>(ws + pl.off_du) + pmine;
+  IO* dxdir = reinterpret_cast<IO*>(ws + pl.off_dxdir) + pmine;
 
   if (w.tid == 0) {
-    for (int i = 0; i < NSTAGE; ++i) mbar_init(&full_bar[i], 1);
+    for (int i = 0; i < NSTAGE_MAIN; ++i) mbar_init(&full_bar[i], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
-  const uint32_t tx_base = (uint32_t)(CK * bw * ESZ * 2 + CK * bw * 4 + CK * NBC * 4 + TILE_FLOATS * 4 + ncs * 4 +
-                                      (WIN ? CK * bw * ESZ + CK * bw * 4 : 0));
+  const uint32_t tx_base = (uint32_t)(CK * CH * ESZ * 2 + CK * CH * 4 + CK * NBC * 4 + TILE_FLOATS * 4 + ncs * 4 +
+                                      (WIN ? CK * CH * ESZ + CK * CH * 4 : 0));
   // chunks are visited last to first: the i-th visited chunk is c = nchunk-1-i
   auto issue = [&](int i) {
-    const int st = i % NSTAGE;
+    const int st = i % NSTAGE_MAIN;
     const int c = nchunk - 1 - i;
     uint8_t* sm = smem + st * St::BYTES;
     const int64_t tc = t0 + (int64_t)c * CK;
-    const int64_t row = (int64_t)b * pl.T + tc;
+    const int64_t row = (int64_t)b * T + tc;
     const int64_t cc = (int64_t)b * pl.NC + tc / CK;
-    const int64_t row2 = row + pl.tbar;          // first token leaving the window of this chunk's tokens
+    const int64_t row2 = row + tbar;             // first token leaving the window of this chunk's tokens
     const bool win_rows = WIN && row2 < BT;      // its B/C rows exist (else no token of the chunk has t + Tbar < T)
     mbar_expect_tx(&full_bar[st], tx_base + (win_rows ? CK * NBC * 4 : 0));
     tma_2d(sm + St::X, &tmX, tile * CH, row, &full_bar[st]);
@@ -556,14 +561,14 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     bulk_1d(sm + St::CS, cs + cc * P + tile * CH, ncs * 4, &full_bar[st]);
     if (WIN) {
       // rows of the tokens leaving the window; past the end of the whole tensor TMA fills zeros, and rows
-      // that belong to the next batch element are never used (guarded by t + Tbar < T)
+      // that belong to the next batch element are masked out below (t + Tbar < T fails)
       tma_2d(sm + St::G2, &tmG, tile * CH, row2, &full_bar[st]);
       tma_2d(sm + St::D2, &tmD, tile * CH, row2, &full_bar[st]);
       if (win_rows) bulk_1d(sm + St::BC2, bc + row2 * NBC, CK * NBC * 4, &full_bar[st]);
     }
   };
   if (w.tid == 0)
-    for (int i = 0; i < NSTAGE && i < nchunk; ++i) issue(i);
+    for (int i = 0; i < NSTAGE_MAIN && i < nchunk; ++i) issue(i);
 
   u64 A2[8], mu[8], dAacc[8];
   load_A2(A_log, w, A2);
@@ -592,18 +597,27 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     sw[0] = swp[0]; sw[1] = swp[1];
   }
   float dbacc = 0.f;
-  const int pmine = w.pa + w.half;   // the channel whose per-token outputs this lane finalises
 
   for (int i = 0; i < nchunk; ++i) {
-    const int st = i % NSTAGE;
+    const int st = i % NSTAGE_MAIN;
     const int c = nchunk - 1 - i;
-    const uint8_t* sm = smem + st * St::BYTES;
-    const bool ok = mbar_wait(&full_bar[st], (i / NSTAGE) & 1);
+    uint8_t* sm = smem + st * St::BYTES;
+    const bool ok = mbar_wait(&full_bar[st], (i / NSTAGE_MAIN) & 1);
     const int64_t tc = t0 + (int64_t)c * CK;
     const int nt = (int)min((int64_t)CK, t1 - tc);
     const int rb = i & 1;
+    const int nwin = WIN ? (int)max((int64_t)0, min((int64_t)CK, T - tbar - tc)) : 0;   // tokens j < nwin have t + Tbar < T
     // window Delta sum: fp64 value at the chunk's last token + an fp32 running offset inside the chunk
-    float swc[2] = {(float)sw[0], (float)sw[1]}, swl[2] = {0.f, 0.f};
+    const float swc[2] = {(float)sw[0], (float)sw[1]};
+    float swl[2] = {0.f, 0.f};
+    if (nt < CK) {   // only the last chunk of a sequence: neutralise the slots past its end
+      if (ok) {
+        zero_rows(sm + St::D, CH * 4, nt, w.tid);
+        zero_rows(sm + St::G, CH * ESZ, nt, w.tid);
+        zero_rows(sm + St::BC, NBC * 4, nt, w.tid);
+      }
+      __syncthreads();
+    }
     if (ok) {
       // state at the chunk start: local checkpoint + decayed true segment-start state
       u64 h[8];
@@ -619,148 +633,146 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
           h[2 * q + 1] = fma2(ex2_2(mul2(c2[q / 2], A2[2 * q + 1])), hq.y, h[2 * q + 1]);
         }
       }
-      // forward rebuild of the chunk
-      u64 hs[CK][8];
+      // forward rebuild: states after tokens 0, 2, 4, 6
+      u64 hs[CK / 2][8];
 #pragma unroll
-      for (int j = 0; j < CK; ++j) {
-        if (j < nt) {
-          const float2 dv = lds_pair<float>(sm + St::D, j, w.k);
-          const float2 xv = lds_pair<IO>(sm + St::X, j, w.k);
-          const float* brow = reinterpret_cast<const float*>(sm + St::BC) + j * NBC + 8 * w.half;
-          const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
-          const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
-          const u64 Bp[4] = {b01.x, b01.y, b23.x, b23.y};
-          const u64 d2[2] = {pk(dv.x, dv.x), pk(dv.y, dv.y)};
-          const u64 dx2[2] = {pk(dv.x * xv.x, dv.x * xv.x), pk(dv.y * xv.y, dv.y * xv.y)};
+      for (int j = 0; j < CK - 1; ++j) {
+        __syncwarp();   // keeps the staged loads of later tokens from being hoisted (register pressure)
+        const float2 dv = lds_pair<float>(sm + St::D, j, w.k);
+        const float2 xv = lds_pair<IO>(sm + St::X, j, w.k);
+        const float* brow = reinterpret_cast<const float*>(sm + St::BC) + j * NBC + 8 * w.half;
+        const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
+        const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
+        const u64 Bp[4] = {b01.x, b01.y, b23.x, b23.y};
+        const u64 d2[2] = {pk(dv.x, dv.x), pk(dv.y, dv.y)};
+        const u64 dx2[2] = {pk(dv.x * xv.x, dv.x * xv.x), pk(dv.y * xv.y, dv.y * xv.y)};
 #pragma unroll
-          for (int u = 0; u < 8; ++u) h[u] = fma2(ex2_2(mul2(d2[u / 4], A2[u])), h[u], mul2(dx2[u / 4], Bp[u % 4]));
+        for (int u = 0; u < 8; ++u) h[u] = fma2(ex2_2(mul2(d2[u / 4], A2[u])), h[u], mul2(dx2[u / 4], Bp[u % 4]));
+        if ((j & 1) == 0) {
+#pragma unroll
+          for (int u = 0; u < 8; ++u) hs[j / 2][u] = h[u];
         }
-#pragma unroll
-        for (int u = 0; u < 8; ++u) hs[j][u] = h[u];
       }
-      // reverse walk
+      // backward walk
 #pragma unroll
       for (int j = CK - 1; j >= 0; --j) {
-        if (j < nt) {
-          const int64_t t = tc + j;
-          const float2 dv = lds_pair<float>(sm + St::D, j, w.k);
-          const float2 xv = lds_pair<IO>(sm + St::X, j, w.k);
-          const float2 gv = lds_pair<IO>(sm + St::G, j, w.k);
-          const float* brow = reinterpret_cast<const float*>(sm + St::BC) + j * NBC + 8 * w.half;
-          const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
-          const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
-          const ulonglong2 c01 = *reinterpret_cast<const ulonglong2*>(brow + NS);
-          const ulonglong2 c23 = *reinterpret_cast<const ulonglong2*>(brow + NS + 4);
-          const u64 Bp[4] = {b01.x, b01.y, b23.x, b23.y};
-          const u64 Cp[4] = {c01.x, c01.y, c23.x, c23.y};
-          const float dd[2] = {dv.x, dv.y}, xs[2] = {xv.x, xv.y}, gs[2] = {gv.x, gv.y};
-          const float dxs[2] = {dv.x * xv.x, dv.y * xv.y};
-          // mu_i += g_i C_i   (mu already carries abar_{i+1} mu_{i+1})
+        __syncwarp();
+        const float2 dv = lds_pair<float>(sm + St::D, j, w.k);
+        const float2 xv = lds_pair<IO>(sm + St::X, j, w.k);
+        const float2 gv = lds_pair<IO>(sm + St::G, j, w.k);
+        const float* brow = reinterpret_cast<const float*>(sm + St::BC) + j * NBC + 8 * w.half;
+        const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
+        const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
+        const ulonglong2 c01 = *reinterpret_cast<const ulonglong2*>(brow + NS);
+        const ulonglong2 c23 = *reinterpret_cast<const ulonglong2*>(brow + NS + 4);
+        const u64 Bp[4] = {b01.x, b01.y, b23.x, b23.y};
+        const u64 Cp[4] = {c01.x, c01.y, c23.x, c23.y};
+        const float dd[2] = {dv.x, dv.y}, xs[2] = {xv.x, xv.y}, gs[2] = {gv.x, gv.y};
+        const float dxs[2] = {dv.x * xv.x, dv.y * xv.y};
+        const u64 d2[2] = {pk(dd[0], dd[0]), pk(dd[1], dd[1])};
+        const u64 dx2[2] = {pk(dxs[0], dxs[0]), pk(dxs[1], dxs[1])};
+        const u64 g2[2] = {pk(gs[0], gs[0]), pk(gs[1], gs[1])};
+        // mu_i += g_i C_i   (mu already carries abar_{i+1} mu_{i+1})
 #pragma unroll
-          for (int u = 0; u < 8; ++u) mu[u] = fma2(pk(gs[u / 4], gs[u / 4]), Cp[u % 4], mu[u]);
-          if (WIN) {
-            const int64_t t2 = t + pl.tbar;
-            if (t2 < pl.T) {
-              // exact exit of token t2 from the window: subtract W_i gC_{t2}, W_i = exp(A * sum_{j=i+1..t2} Delta_j)
-              const float2 d2v = lds_pair<float>(sm + St::D2, j, w.k);
-              const float2 g2v = lds_pair<IO>(sm + St::G2, j, w.k);
-              const float swf[2] = {swc[0] + swl[0], swc[1] + swl[1]};
-              // skip when every factor W = 2^(A2 * sum) of the warp is below 2^-64: the term is then far
-              // below one rounding unit of mu
-              const bool live = w.act && (swf[0] * a2max[0] > -64.f || swf[1] * a2max[1] > -64.f);
-              if (__any_sync(0xffffffffu, live)) {
-                const float* crow = reinterpret_cast<const float*>(sm + St::BC2) + j * NBC + NS + 8 * w.half;
-                const ulonglong2 e01 = *reinterpret_cast<const ulonglong2*>(crow);
-                const ulonglong2 e23 = *reinterpret_cast<const ulonglong2*>(crow + 4);
-                const u64 C2p[4] = {e01.x, e01.y, e23.x, e23.y};
-                const float g2s[2] = {-g2v.x, -g2v.y};
+        for (int u = 0; u < 8; ++u) mu[u] = fma2(g2[u / 4], Cp[u % 4], mu[u]);
+        if (WIN) {
+          // exact exit of token t2 = t + Tbar from the window: subtract W_i gC_{t2},
+          // W_i = exp(A * sum_{j=i+1..t2} Delta_j); masked out when t2 >= T
+          const float wm = j < nwin ? 1.f : 0.f;
+          float2 d2v = lds_pair<float>(sm + St::D2, j, w.k);
+          d2v.x *= wm; d2v.y *= wm;
+          const float swf[2] = {swc[0] + swl[0], swc[1] + swl[1]};
+          // skip when every factor W = 2^(A2 * sum) of the warp is below 2^-64: the term is then far
+          // below one rounding unit of mu
+          const bool live = j < nwin && w.act && (swf[0] * a2max[0] > -64.f || swf[1] * a2max[1] > -64.f);
+          if (__any_sync(0xffffffffu, live)) {
+            const float2 g2v = lds_pair<IO>(sm + St::G2, j, w.k);
+            const float* crow = reinterpret_cast<const float*>(sm + St::BC2) + j * NBC + NS + 8 * w.half;
+            const ulonglong2 e01 = *reinterpret_cast<const ulonglong2*>(crow);
+            const ulonglong2 e23 = *reinterpret_cast<const ulonglong2*>(crow + 4);
+            const u64 C2p[4] = {e01.x, e01.y, e23.x, e23.y};
+            const u64 ng2[2] = {pk(-g2v.x, -g2v.x), pk(-g2v.y, -g2v.y)};
+            const u64 sw2[2] = {pk(swf[0], swf[0]), pk(swf[1], swf[1])};
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                  const u64 W = ex2_2(mul2(pk(swf[u / 4], swf[u / 4]), A2[u]));
-                  mu[u] = fma2(W, mul2(pk(g2s[u / 4], g2s[u / 4]), C2p[u % 4]), mu[u]);
-                }
-              }
-              swl[0] += dd[0] - d2v.x;   // window of token t-1: (t-1, t-1+Tbar]
-              swl[1] += dd[1] - d2v.y;
-            } else {
-              swl[0] += dd[0];           // token t+Tbar does not exist: the (clipped) window sum only grows
-              swl[1] += dd[1];
-            }
+            for (int u = 0; u < 8; ++u)
+              mu[u] = fma2(ex2_2(mul2(sw2[u / 4], A2[u])), mul2(ng2[u / 4], C2p[u % 4]), mu[u]);
           }
-          u64 vB[4], vC[4];
-          float ssum[2], dsum[2];
-#pragma unroll
-          for (int ch = 0; ch < 2; ++ch) {
-            const u64 d2 = pk(dd[ch], dd[ch]), dx2 = pk(dxs[ch], dxs[ch]), ndx2 = pk(-dxs[ch], -dxs[ch]);
-            const u64 g2 = pk(gs[ch], gs[ch]);
-            u64 sacc = 0ull, dacc = 0ull;
-#pragma unroll
-            for (int m = 0; m < 4; ++m) {
-              const int u = ch * 4 + m;
-              const u64 hn = hs[j][u];
-              vB[m] = ch == 0 ? mul2(mu[u], dx2) : fma2(mu[u], dx2, vB[m]);   // dB partial (two channels)
-              vC[m] = ch == 0 ? mul2(g2, hn) : fma2(g2, hn, vC[m]);           // dC partial
-              sacc = fma2(mu[u], Bp[m], sacc);
-              const u64 hb = fma2(ndx2, Bp[m], hn);                            // abar_i h_{i-1}
-              const u64 q = mul2(mu[u], hb);
-              dacc = fma2(q, A2[u], dacc);
-              dAacc[u] = fma2(q, d2, dAacc[u]);
-              mu[u] = mul2(mu[u], ex2_2(mul2(d2, A2[u])));                     // ready for token i-1
-            }
-            ssum[ch] = hsum(sacc);
-            dsum[ch] = hsum(dacc);
-          }
-#pragma unroll
-          for (int ch = 0; ch < 2; ++ch) {
-            ssum[ch] += __shfl_xor_sync(0xffffffffu, ssum[ch], 1);
-            dsum[ch] += __shfl_xor_sync(0xffffffffu, dsum[ch], 1);
-          }
-          {
-            const float d = w.half ? dd[1] : dd[0], xx = w.half ? xs[1] : xs[0];
-            const float sv = w.half ? ssum[1] : ssum[0], dsv = w.half ? dsum[1] : dsum[0];
-            const float ddelta = fmaf(dsv, LN2, xx * sv);
-            const float duv = ddelta * sig_from_delta(d);
-            dbacc += duv;
-            if (w.act) {
-              const int64_t row = (int64_t)b * pl.T + t;
-              st_io<IO>(du + row * pl.du_ld + pmine, duv);
-              st_io<IO>(dxdir + row * P + pmine, d * sv);
-            }
-          }
-          // transposing reduction over the 16 lanes of equal parity: afterwards this lane holds the warp total of
-          // value (lane >> 1): values 0..7 = dB[8*half + .], 8..15 = dC[8*half + .]
-          float v[16];
-#pragma unroll
-          for (int m = 0; m < 4; ++m) { upk(vB[m], v[2 * m], v[2 * m + 1]); upk(vC[m], v[8 + 2 * m], v[8 + 2 * m + 1]); }
-#pragma unroll
-          for (int off = 16, cnt = 8; cnt >= 1; off >>= 1, cnt >>= 1) {
-            const bool up = (lane & off) != 0;
-#pragma unroll
-            for (int k = 0; k < cnt; ++k) {
-              const float send = up ? v[k] : v[k + cnt];
-              const float keep = up ? v[k + cnt] : v[k];
-              v[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
-            }
-          }
-          const int vi = lane >> 1;
-          red[rb][warp][j][(vi & 8) * 2 + 8 * w.half + (vi & 7)] = v[0];
+          swl[0] += dd[0] - d2v.x;   // window of token t-1: (t-1, t-1+Tbar]
+          swl[1] += dd[1] - d2v.y;
         }
+        u64 vB[4], vC[4];
+        float ssum[2], dsum[2];
+#pragma unroll
+        for (int ch = 0; ch < 2; ++ch) {
+          u64 sacc = 0ull, dacc = 0ull;
+#pragma unroll
+          for (int m = 0; m < 4; ++m) {
+            const int u = ch * 4 + m;
+            const u64 a = ex2_2(mul2(d2[ch], A2[u]));
+            const u64 bx = mul2(dx2[ch], Bp[m]);
+            u64 hn, hb;                                        // h_i and abar_i h_{i-1}
+            if (j & 1) { hb = mul2(a, hs[j / 2][u]); hn = fma2(a, hs[j / 2][u], bx); }
+            else { hn = hs[j / 2][u]; hb = fma2(bx, pk(-1.f, -1.f), hn); }
+            vB[m] = ch == 0 ? mul2(mu[u], dx2[ch]) : fma2(mu[u], dx2[ch], vB[m]);   // dB partial (two channels)
+            vC[m] = ch == 0 ? mul2(g2[ch], hn) : fma2(g2[ch], hn, vC[m]);           // dC partial
+            sacc = fma2(mu[u], Bp[m], sacc);
+            const u64 q = mul2(mu[u], hb);
+            dacc = fma2(q, A2[u], dacc);
+            dAacc[u] = fma2(q, d2[ch], dAacc[u]);
+            mu[u] = mul2(mu[u], a);                                                  // ready for token i-1
+          }
+          ssum[ch] = hsum(sacc);
+          dsum[ch] = hsum(dacc);
+        }
+#pragma unroll
+        for (int ch = 0; ch < 2; ++ch) {
+          ssum[ch] += __shfl_xor_sync(0xffffffffu, ssum[ch], 1);
+          dsum[ch] += __shfl_xor_sync(0xffffffffu, dsum[ch], 1);
+        }
+        {
+          const float d = w.half ? dd[1] : dd[0], xx = w.half ? xs[1] : xs[0];
+          const float sv = w.half ? ssum[1] : ssum[0], dsv = w.half ? dsum[1] : dsum[0];
+          const float ddelta = fmaf(dsv, LN2, xx * sv);
+          const float duv = ddelta * sig_from_delta(d);
+          dbacc += duv;
+          if (w.act && j < nt) {
+            const int64_t row = (int64_t)b * T + tc + j;
+            st_io<IO>(du + row * du_ld, duv);
+            st_io<IO>(dxdir + row * P, d * sv);
+          }
+        }
+        // transposing reduction over the 16 lanes of equal parity: afterwards this lane holds the warp total of
+        // value (lane >> 1): values 0..7 = dB[8*half + .], 8..15 = dC[8*half + .]
+        float v[16];
+#pragma unroll
+        for (int m = 0; m < 4; ++m) { upk(vB[m], v[2 * m], v[2 * m + 1]); upk(vC[m], v[8 + 2 * m], v[8 + 2 * m + 1]); }
+#pragma unroll
+        for (int off = 16, cnt = 8; cnt >= 1; off >>= 1, cnt >>= 1) {
+          const bool up = (lane & off) != 0;
+#pragma unroll
+          for (int k = 0; k < cnt; ++k) {
+            const float send = up ? v[k] : v[k + cnt];
+            const float keep = up ? v[k + cnt] : v[k];
+            v[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+          }
+        }
+        const int vi = lane >> 1;
+        red[rb][warp][j][(vi & 8) * 2 + 8 * w.half + (vi & 7)] = v[0];
       }
     }
     if (WIN) { sw[0] += (double)swl[0]; sw[1] += (double)swl[1]; }
-    (void)swc;
     const int bad = __syncthreads_or(ok ? 0 : 1);
     if (bad) {
       if (w.tid == 0) atomicExch(status, AS_ERR_TIMEOUT);
       return;
     }
-    if (w.tid == 0 && i + NSTAGE < nchunk) issue(i + NSTAGE);
+    if (w.tid == 0 && i + NSTAGE_MAIN < nchunk) issue(i + NSTAGE_MAIN);
     for (int e = w.tid; e < nt * NBC; e += CH) {
       const int j = e / NBC, q = e % NBC;
       float sum = 0.f;
 #pragma unroll
       for (int wq = 0; wq < CH / 32; ++wq) sum += red[rb][wq][j][q];
-      atomicAdd(dbc + ((int64_t)b * pl.T + tc + j) * NBC + q, sum);
+      atomicAdd(dbc + ((int64_t)b * T + tc + j) * NBC + q, sum);
     }
   }
   if (w.act) {
@@ -845,7 +857,7 @@ int launch_main_t(const Plan& pl, const ScanPtrs& sp, float* dA_log, float* db_d
   Maps m;
   if (make_maps(pl, sp, &m)) return 1;
   using St = Stage<sizeof(IO), true, true, !FULL>;
-  const int bytes = NSTAGE * St::BYTES + 128;
+  const int bytes = NSTAGE_MAIN * St::BYTES + 128;
   auto kern = adjoint_main_kernel<IO, FULL>;
   static bool once = false;
   if (!once) { if (set_smem(kern, bytes)) return 1; once = true; }
