@@ -155,6 +155,7 @@ struct Stage {
   static constexpr int BYTES = BC2 + (WIN ? CK * NBC * 4 : 0);
 };
 constexpr int NSTAGE = 3;        // ascending kernels
+constexpr int HALF = CK / 2;       // tokens per unrolled loop body of the main adjoint kernel
 constexpr int NSTAGE_MAIN = 2;   // main adjoint kernel: a chunk takes thousands of cycles, one chunk of lookahead suffices
 
 template <typename IO> __device__ __forceinline__ float2 lds_pair(const uint8_t* tile, int j, int k);
@@ -633,131 +634,155 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
           h[2 * q + 1] = fma2(ex2_2(mul2(c2[q / 2], A2[2 * q + 1])), hq.y, h[2 * q + 1]);
         }
       }
-      // forward rebuild: states after tokens 0, 2, 4, 6
-      u64 hs[CK / 2][8];
+      // forward rebuild in two halves of four tokens (one copy of the code, rolled loop): only the states
+      // after tokens 0, 2, 4, 6 are kept; `cur` holds the pair of the half being processed, `hsA` parks the
+      // first half's pair while the second half is rebuilt and walked.
+      u64 hsA[2][8], cur[2][8];
+#pragma unroll 1
+      for (int k = 0; k < 2; ++k) {
+        const uint8_t* smk = sm + k * HALF * CH * ESZ;          // x rows of this half
+        const uint8_t* smd = sm + St::D + k * HALF * CH * 4;
+        const float* bck = reinterpret_cast<const float*>(sm + St::BC) + k * HALF * NBC + 8 * w.half;
 #pragma unroll
-      for (int j = 0; j < CK - 1; ++j) {
-        __syncwarp();   // keeps the staged loads of later tokens from being hoisted (register pressure)
-        const float2 dv = lds_pair<float>(sm + St::D, j, w.k);
-        const float2 xv = lds_pair<IO>(sm + St::X, j, w.k);
-        const float* brow = reinterpret_cast<const float*>(sm + St::BC) + j * NBC + 8 * w.half;
-        const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
-        const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
-        const u64 Bp[4] = {b01.x, b01.y, b23.x, b23.y};
-        const u64 d2[2] = {pk(dv.x, dv.x), pk(dv.y, dv.y)};
-        const u64 dx2[2] = {pk(dv.x * xv.x, dv.x * xv.x), pk(dv.y * xv.y, dv.y * xv.y)};
+        for (int jj = 0; jj < HALF; ++jj) {
+          if (jj == HALF - 1 && k == 1) break;                  // the state after the chunk's last token is rebuilt below
+          __syncwarp();   // keeps the staged loads of later tokens from being hoisted (register pressure)
+          const float2 dv = lds_pair<float>(smd, jj, w.k);
+          const float2 xv = lds_pair<IO>(smk + St::X, jj, w.k);
+          const float* brow = bck + jj * NBC;
+          const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
+          const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
+          const u64 Bp[4] = {b01.x, b01.y, b23.x, b23.y};
+          const u64 d2[2] = {pk(dv.x, dv.x), pk(dv.y, dv.y)};
+          const u64 dx2[2] = {pk(dv.x * xv.x, dv.x * xv.x), pk(dv.y * xv.y, dv.y * xv.y)};
 #pragma unroll
-        for (int u = 0; u < 8; ++u) h[u] = fma2(ex2_2(mul2(d2[u / 4], A2[u])), h[u], mul2(dx2[u / 4], Bp[u % 4]));
-        if ((j & 1) == 0) {
+          for (int u = 0; u < 8; ++u) h[u] = fma2(ex2_2(mul2(d2[u / 4], A2[u])), h[u], mul2(dx2[u / 4], Bp[u % 4]));
+          if ((jj & 1) == 0) {
 #pragma unroll
-          for (int u = 0; u < 8; ++u) hs[j / 2][u] = h[u];
+            for (int u = 0; u < 8; ++u) cur[jj / 2][u] = h[u];
+          }
+        }
+        if (k == 0) {
+#pragma unroll
+          for (int u = 0; u < 8; ++u) { hsA[0][u] = cur[0][u]; hsA[1][u] = cur[1][u]; }
         }
       }
-      // backward walk
+      // backward walk, second half first
+#pragma unroll 1
+      for (int k = 1; k >= 0; --k) {
+        if (k == 0) {
 #pragma unroll
-      for (int j = CK - 1; j >= 0; --j) {
-        __syncwarp();
-        const float2 dv = lds_pair<float>(sm + St::D, j, w.k);
-        const float2 xv = lds_pair<IO>(sm + St::X, j, w.k);
-        const float2 gv = lds_pair<IO>(sm + St::G, j, w.k);
-        const float* brow = reinterpret_cast<const float*>(sm + St::BC) + j * NBC + 8 * w.half;
-        const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
-        const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
-        const ulonglong2 c01 = *reinterpret_cast<const ulonglong2*>(brow + NS);
-        const ulonglong2 c23 = *reinterpret_cast<const ulonglong2*>(brow + NS + 4);
-        const u64 Bp[4] = {b01.x, b01.y, b23.x, b23.y};
-        const u64 Cp[4] = {c01.x, c01.y, c23.x, c23.y};
-        const float dd[2] = {dv.x, dv.y}, xs[2] = {xv.x, xv.y}, gs[2] = {gv.x, gv.y};
-        const float dxs[2] = {dv.x * xv.x, dv.y * xv.y};
-        const u64 d2[2] = {pk(dd[0], dd[0]), pk(dd[1], dd[1])};
-        const u64 dx2[2] = {pk(dxs[0], dxs[0]), pk(dxs[1], dxs[1])};
-        const u64 g2[2] = {pk(gs[0], gs[0]), pk(gs[1], gs[1])};
-        // mu_i += g_i C_i   (mu already carries abar_{i+1} mu_{i+1})
+          for (int u = 0; u < 8; ++u) { cur[0][u] = hsA[0][u]; cur[1][u] = hsA[1][u]; }
+        }
+        const uint8_t* smk = sm + k * HALF * CH * ESZ;          // x / dy rows of this half
+        const uint8_t* smd = sm + k * HALF * CH * 4;            // Delta rows
+        const float* bck = reinterpret_cast<const float*>(sm) + k * HALF * NBC + 8 * w.half;
 #pragma unroll
-        for (int u = 0; u < 8; ++u) mu[u] = fma2(g2[u / 4], Cp[u % 4], mu[u]);
-        if (WIN) {
-          // exact exit of token t2 = t + Tbar from the window: subtract W_i gC_{t2},
-          // W_i = exp(A * sum_{j=i+1..t2} Delta_j); masked out when t2 >= T
-          const float wm = j < nwin ? 1.f : 0.f;
-          float2 d2v = lds_pair<float>(sm + St::D2, j, w.k);
-          d2v.x *= wm; d2v.y *= wm;
-          const float swf[2] = {swc[0] + swl[0], swc[1] + swl[1]};
-          // skip when every factor W = 2^(A2 * sum) of the warp is below 2^-64: the term is then far
-          // below one rounding unit of mu
-          const bool live = j < nwin && w.act && (swf[0] * a2max[0] > -64.f || swf[1] * a2max[1] > -64.f);
-          if (__any_sync(0xffffffffu, live)) {
-            const float2 g2v = lds_pair<IO>(sm + St::G2, j, w.k);
-            const float* crow = reinterpret_cast<const float*>(sm + St::BC2) + j * NBC + NS + 8 * w.half;
-            const ulonglong2 e01 = *reinterpret_cast<const ulonglong2*>(crow);
-            const ulonglong2 e23 = *reinterpret_cast<const ulonglong2*>(crow + 4);
-            const u64 C2p[4] = {e01.x, e01.y, e23.x, e23.y};
-            const u64 ng2[2] = {pk(-g2v.x, -g2v.x), pk(-g2v.y, -g2v.y)};
-            const u64 sw2[2] = {pk(swf[0], swf[0]), pk(swf[1], swf[1])};
+        for (int jj = HALF - 1; jj >= 0; --jj) {
+          const int j = k * HALF + jj;
+          __syncwarp();
+          const float2 dv = lds_pair<float>(smd + St::D, jj, w.k);
+          const float2 xv = lds_pair<IO>(smk + St::X, jj, w.k);
+          const float2 gv = lds_pair<IO>(smk + St::G, jj, w.k);
+          const float* brow = bck + St::BC / 4 + jj * NBC;
+          const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
+          const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
+          const ulonglong2 c01 = *reinterpret_cast<const ulonglong2*>(brow + NS);
+          const ulonglong2 c23 = *reinterpret_cast<const ulonglong2*>(brow + NS + 4);
+          const u64 Bp[4] = {b01.x, b01.y, b23.x, b23.y};
+          const u64 Cp[4] = {c01.x, c01.y, c23.x, c23.y};
+          const float dd[2] = {dv.x, dv.y}, xs[2] = {xv.x, xv.y}, gs[2] = {gv.x, gv.y};
+          const float dxs[2] = {dv.x * xv.x, dv.y * xv.y};
+          const u64 d2[2] = {pk(dd[0], dd[0]), pk(dd[1], dd[1])};
+          const u64 dx2[2] = {pk(dxs[0], dxs[0]), pk(dxs[1], dxs[1])};
+          const u64 g2[2] = {pk(gs[0], gs[0]), pk(gs[1], gs[1])};
+          // mu_i += g_i C_i   (mu already carries abar_{i+1} mu_{i+1})
 #pragma unroll
-            for (int u = 0; u < 8; ++u)
-              mu[u] = fma2(ex2_2(mul2(sw2[u / 4], A2[u])), mul2(ng2[u / 4], C2p[u % 4]), mu[u]);
+          for (int u = 0; u < 8; ++u) mu[u] = fma2(g2[u / 4], Cp[u % 4], mu[u]);
+          if (WIN) {
+            // exact exit of token t2 = t + Tbar from the window: subtract W_i gC_{t2},
+            // W_i = exp(A * sum_{j=i+1..t2} Delta_j); masked out when t2 >= T
+            const float wm = j < nwin ? 1.f : 0.f;
+            float2 d2v = lds_pair<float>(smd + St::D2, jj, w.k);
+            d2v.x *= wm; d2v.y *= wm;
+            const float swf[2] = {swc[0] + swl[0], swc[1] + swl[1]};
+            // skip when every factor W = 2^(A2 * sum) of the warp is below 2^-64: the term is then far
+            // below one rounding unit of mu
+            const bool live = j < nwin && w.act && (swf[0] * a2max[0] > -64.f || swf[1] * a2max[1] > -64.f);
+            if (__any_sync(0xffffffffu, live)) {
+              const float2 g2v = lds_pair<IO>(smk + St::G2, jj, w.k);
+              const float* crow = bck + St::BC2 / 4 + jj * NBC + NS;
+              const ulonglong2 e01 = *reinterpret_cast<const ulonglong2*>(crow);
+              const ulonglong2 e23 = *reinterpret_cast<const ulonglong2*>(crow + 4);
+              const u64 C2p[4] = {e01.x, e01.y, e23.x, e23.y};
+              const u64 ng2[2] = {pk(-g2v.x, -g2v.x), pk(-g2v.y, -g2v.y)};
+              const u64 sw2[2] = {pk(swf[0], swf[0]), pk(swf[1], swf[1])};
+#pragma unroll
+              for (int u = 0; u < 8; ++u)
+                mu[u] = fma2(ex2_2(mul2(sw2[u / 4], A2[u])), mul2(ng2[u / 4], C2p[u % 4]), mu[u]);
+            }
+            swl[0] += dd[0] - d2v.x;   // window of token t-1: (t-1, t-1+Tbar]
+            swl[1] += dd[1] - d2v.y;
           }
-          swl[0] += dd[0] - d2v.x;   // window of token t-1: (t-1, t-1+Tbar]
-          swl[1] += dd[1] - d2v.y;
-        }
-        u64 vB[4], vC[4];
-        float ssum[2], dsum[2];
+          u64 vB[4], vC[4];
+          float ssum[2], dsum[2];
 #pragma unroll
-        for (int ch = 0; ch < 2; ++ch) {
-          u64 sacc = 0ull, dacc = 0ull;
+          for (int ch = 0; ch < 2; ++ch) {
+            u64 sacc = 0ull, dacc = 0ull;
 #pragma unroll
-          for (int m = 0; m < 4; ++m) {
-            const int u = ch * 4 + m;
-            const u64 a = ex2_2(mul2(d2[ch], A2[u]));
-            const u64 bx = mul2(dx2[ch], Bp[m]);
-            u64 hn, hb;                                        // h_i and abar_i h_{i-1}
-            if (j & 1) { hb = mul2(a, hs[j / 2][u]); hn = fma2(a, hs[j / 2][u], bx); }
-            else { hn = hs[j / 2][u]; hb = fma2(bx, pk(-1.f, -1.f), hn); }
-            vB[m] = ch == 0 ? mul2(mu[u], dx2[ch]) : fma2(mu[u], dx2[ch], vB[m]);   // dB partial (two channels)
-            vC[m] = ch == 0 ? mul2(g2[ch], hn) : fma2(g2[ch], hn, vC[m]);           // dC partial
-            sacc = fma2(mu[u], Bp[m], sacc);
-            const u64 q = mul2(mu[u], hb);
-            dacc = fma2(q, A2[u], dacc);
-            dAacc[u] = fma2(q, d2[ch], dAacc[u]);
-            mu[u] = mul2(mu[u], a);                                                  // ready for token i-1
+            for (int m = 0; m < 4; ++m) {
+              const int u = ch * 4 + m;
+              const u64 a = ex2_2(mul2(d2[ch], A2[u]));
+              const u64 bx = mul2(dx2[ch], Bp[m]);
+              u64 hn, hb;                                        // h_i and abar_i h_{i-1}
+              if (jj & 1) { hb = mul2(a, cur[jj / 2][u]); hn = fma2(a, cur[jj / 2][u], bx); }
+              else { hn = cur[jj / 2][u]; hb = fma2(bx, pk(-1.f, -1.f), hn); }
+              vB[m] = ch == 0 ? mul2(mu[u], dx2[ch]) : fma2(mu[u], dx2[ch], vB[m]);   // dB partial (two channels)
+              vC[m] = ch == 0 ? mul2(g2[ch], hn) : fma2(g2[ch], hn, vC[m]);           // dC partial
+              sacc = fma2(mu[u], Bp[m], sacc);
+              const u64 q = mul2(mu[u], hb);
+              dacc = fma2(q, A2[u], dacc);
+              dAacc[u] = fma2(q, d2[ch], dAacc[u]);
+              mu[u] = mul2(mu[u], a);                                                  // ready for token i-1
+            }
+            ssum[ch] = hsum(sacc);
+            dsum[ch] = hsum(dacc);
           }
-          ssum[ch] = hsum(sacc);
-          dsum[ch] = hsum(dacc);
-        }
 #pragma unroll
-        for (int ch = 0; ch < 2; ++ch) {
-          ssum[ch] += __shfl_xor_sync(0xffffffffu, ssum[ch], 1);
-          dsum[ch] += __shfl_xor_sync(0xffffffffu, dsum[ch], 1);
-        }
-        {
-          const float d = w.half ? dd[1] : dd[0], xx = w.half ? xs[1] : xs[0];
-          const float sv = w.half ? ssum[1] : ssum[0], dsv = w.half ? dsum[1] : dsum[0];
-          const float ddelta = fmaf(dsv, LN2, xx * sv);
-          const float duv = ddelta * sig_from_delta(d);
-          dbacc += duv;
-          if (w.act && j < nt) {
-            const int64_t row = (int64_t)b * T + tc + j;
-            st_io<IO>(du + row * du_ld, duv);
-            st_io<IO>(dxdir + row * P, d * sv);
+          for (int ch = 0; ch < 2; ++ch) {
+            ssum[ch] += __shfl_xor_sync(0xffffffffu, ssum[ch], 1);
+            dsum[ch] += __shfl_xor_sync(0xffffffffu, dsum[ch], 1);
           }
-        }
-        // transposing reduction over the 16 lanes of equal parity: afterwards this lane holds the warp total of
-        // value (lane >> 1): values 0..7 = dB[8*half + .], 8..15 = dC[8*half + .]
-        float v[16];
-#pragma unroll
-        for (int m = 0; m < 4; ++m) { upk(vB[m], v[2 * m], v[2 * m + 1]); upk(vC[m], v[8 + 2 * m], v[8 + 2 * m + 1]); }
-#pragma unroll
-        for (int off = 16, cnt = 8; cnt >= 1; off >>= 1, cnt >>= 1) {
-          const bool up = (lane & off) != 0;
-#pragma unroll
-          for (int k = 0; k < cnt; ++k) {
-            const float send = up ? v[k] : v[k + cnt];
-            const float keep = up ? v[k + cnt] : v[k];
-            v[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+          {
+            const float d = w.half ? dd[1] : dd[0], xx = w.half ? xs[1] : xs[0];
+            const float sv = w.half ? ssum[1] : ssum[0], dsv = w.half ? dsum[1] : dsum[0];
+            const float ddelta = fmaf(dsv, LN2, xx * sv);
+            const float duv = ddelta * sig_from_delta(d);
+            dbacc += duv;
+            if (w.act && j < nt) {
+              const int64_t row = (int64_t)b * T + tc + j;
+              st_io<IO>(du + row * du_ld, duv);
+              st_io<IO>(dxdir + row * P, d * sv);
+            }
           }
+          // transposing reduction over the 16 lanes of equal parity: afterwards this lane holds the warp total of
+          // value (lane >> 1): values 0..7 = dB[8*half + .], 8..15 = dC[8*half + .]
+          float v[16];
+#pragma unroll
+          for (int m = 0; m < 4; ++m) { upk(vB[m], v[2 * m], v[2 * m + 1]); upk(vC[m], v[8 + 2 * m], v[8 + 2 * m + 1]); }
+#pragma unroll
+          for (int off = 16, cnt = 8; cnt >= 1; off >>= 1, cnt >>= 1) {
+            const bool up = (lane & off) != 0;
+#pragma unroll
+            for (int kk = 0; kk < cnt; ++kk) {
+              const float send = up ? v[kk] : v[kk + cnt];
+              const float keep = up ? v[kk + cnt] : v[kk];
+              v[kk] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+            }
+          }
+          const int vi = lane >> 1;
+          red[rb][warp][j][(vi & 8) * 2 + 8 * w.half + (vi & 7)] = v[0];
         }
-        const int vi = lane >> 1;
-        red[rb][warp][j][(vi & 8) * 2 + 8 * w.half + (vi & 7)] = v[0];
       }
     }
     if (WIN) { sw[0] += (double)swl[0]; sw[1] += (double)swl[1]; }
