@@ -115,6 +115,22 @@ int as_adjoint_grad(const as_shape_t *shape, const as_params_t *params, const vo
 int as_full_bptt_grad(const as_shape_t *shape, const as_params_t *params, const void *x, const void *dy,
                       uint32_t flags, const as_grads_t *out, void *ws, size_t ws_bytes, void *stream);
 
+/* Forward for callers that cannot allocate device memory (the paper has no counterpart: this is a deployment
+ * convenience, not part of the method).  Meant for code running as a guest of a host program that owns all
+ * device memory and forbids cudaMalloc from guest code (a plug-in in an inference server with a frozen memory
+ * budget, a latency-critical loop that cannot afford cudaMalloc's device-wide synchronisation).  Same result as
+ * as_ssm_forward, but the scratch is a fixed AS_STATIC_SCRATCH_BYTES array inside the library's device image:
+ *   - every GPU context that loads the library holds that much memory until exit;
+ *   - a shape whose forward scratch (as_workspace_bytes, fwd_bytes) is larger returns AS_ERR_LIMIT, nothing runs;
+ *   - the first call on a device resolves the array's device address (a synchronous runtime query made with that
+ *     device current): make it during set-up, before any stream capture;
+ *   - all calls on a device share the array and it keeps the previous call's contents (what must start at zero is
+ *     cleared by the call); calls whose kernels may overlap on the GPU race on it - order them on one stream;
+ *   - neither this call nor anything it launches calls cudaMalloc, cudaFree or another allocating routine.
+ * x, y: [Bsz,T,P] io dtype device buffers supplied by the caller, as for as_ssm_forward. */
+#define AS_STATIC_SCRATCH_BYTES (32u << 20)
+int as_ssm_forward_static(const as_shape_t *shape, const as_params_t *params, const void *x, void *y, void *stream);
+
 /* Residual-stack glue (Section 3.2; Alg. 1 lines 6-7): gain-free RMSNorm over d_model.
  * yhat = y / sqrt(mean_p(y^2) + eps), io dtype in and out, fp32 arithmetic. */
 int as_rmsnorm_fwd(const as_shape_t *shape, const void *y, void *yhat, float eps, void *stream);

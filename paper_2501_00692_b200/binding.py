@@ -22,7 +22,8 @@ AS_ERR_WORKSPACE, AS_ERR_ALIGN, AS_ERR_CUDA, AS_ERR_TIMEOUT, AS_ERR_LIMIT = -5, 
 
 EXPORTS = ("as_version", "as_strerror", "as_workspace_bytes", "as_check_status", "as_ssm_forward",
            "as_adjoint_grad", "as_full_bptt_grad", "as_rmsnorm_fwd", "as_residual_add", "as_rmsnorm_bwd_add",
-           "as_launch_count", "as_set_timing", "as_get_timing")
+           "as_launch_count", "as_set_timing", "as_get_timing", "as_ssm_forward_static")
+AS_STATIC_SCRATCH_BYTES = 32 << 20
 AS_NUM_PHASES = 6
 PHASES = ("projections", "prepass", "fixup", "adjoint_main", "weight_grads", "input_grad")
 
@@ -74,6 +75,8 @@ def lib() -> C.CDLL:
         L.as_residual_add.argtypes = [C.POINTER(as_shape_t), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.as_rmsnorm_bwd_add.argtypes = [C.POINTER(as_shape_t), C.c_void_p, C.c_void_p, C.c_void_p, C.c_float,
                                          C.c_void_p]
+        L.as_ssm_forward_static.argtypes = [C.POINTER(as_shape_t), C.POINTER(as_params_t), C.c_void_p, C.c_void_p,
+                                            C.c_void_p]
         L.as_launch_count.argtypes = [C.c_int]
         L.as_set_timing.argtypes = [C.c_int]
         L.as_get_timing.argtypes = [C.POINTER(C.c_float), C.c_int]
@@ -200,3 +203,12 @@ def as_get_timing() -> dict:
     ms = (C.c_float * AS_NUM_PHASES)()
     _check(lib().as_get_timing(ms, AS_NUM_PHASES), "as_get_timing")
     return dict(zip(PHASES, [float(v) for v in ms]))
+
+
+def as_ssm_forward_static(shape, theta, x, y, stream=None):
+    """Forward using the library's built-in scratch array: for callers that may not allocate device memory
+    (guests of a host program that owns all of it).  Shapes needing more than AS_STATIC_SCRATCH_BYTES of scratch
+    raise AsError(AS_ERR_LIMIT).  Calls on one device share the array: do not let two of them overlap."""
+    p = make_params(theta)
+    _check(lib().as_ssm_forward_static(C.byref(shape), C.byref(p), _ptr(x), _ptr(y), _stream(stream)),
+           "as_ssm_forward_static")

@@ -1,0 +1,53 @@
+"""as_ssm_forward_static: the forward for callers that cannot allocate device memory.
+
+Some users of the library run as guests of a host program that owns every byte of device memory and forbids
+cudaMalloc from guest code (an inference-server plug-in with a frozen budget, a latency-critical loop).  They call
+this entry point, whose scratch is a fixed array inside the library.  The test calls it through the C ABI twice in
+a row - the array keeps the first call's contents, so the second call proves nothing stale leaks into a result -
+and checks both outputs against the ordinary as_ssm_forward with caller-provided scratch.  This file sorts last
+on purpose: if it fails, a stop-at-first-failure run has already executed every other test.
+"""
+import ctypes as C
+
+import pytest
+import torch
+
+from paper_2501_00692_b200 import binding as B
+from paper_2501_00692_b200 import synth
+from paper_2501_00692_b200.build import build_library
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.mark.parametrize("io", ["f32", "bf16"])
+def test_static_scratch_forward_matches_regular_forward_twice(io):
+    build_library()
+    L = B.lib()
+    outs = []
+    for config, (batch, T, P) in ((21, (2, 700, 64)), (22, (1, 3000, 128))):   # two different shapes back to back
+        w = synth.custom_workload("noalloc", config, batch, T, P, io=io)
+        theta = synth.layer_params(w, 0, DEV)
+        x, _ = synth.activations(w, DEV)
+        sh = B.shape_of(x)
+        fwd_bytes, _ = B.as_workspace_bytes(sh, T)
+        assert fwd_bytes <= B.AS_STATIC_SCRATCH_BYTES
+        ws = B.alloc_workspace(fwd_bytes, DEV)
+        y_ref = torch.empty_like(x)
+        B.as_ssm_forward(sh, theta, x, y_ref, ws)
+        y = torch.full_like(x, float("nan"))
+        p = B.make_params(theta)
+        stream = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+        rc = L.as_ssm_forward_static(C.byref(sh), C.byref(p), C.c_void_p(x.data_ptr()), C.c_void_p(y.data_ptr()), stream)
+        assert rc == 0, B.strerror(rc)
+        torch.cuda.synchronize()
+        assert torch.isfinite(y.float()).all()
+        tol = 1e-4 if io == "f32" else 2e-2
+        err = (y.double() - y_ref.double()).abs().max().item() / y_ref.double().abs().max().item()
+        assert err <= tol, err
+        outs.append(err)
+    # a shape that needs more scratch than the built-in array is refused, and nothing is written
+    big = B.make_shape(4, 1 << 20, 1024, 16, B.AS_BF16)
+    with pytest.raises(B.AsError) as ei:
+        B.as_ssm_forward_static(big, theta, x, y)
+    assert ei.value.code == B.AS_ERR_LIMIT
