@@ -79,6 +79,22 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def max_over_ranks(values, device, world):
+    """Element-wise maximum over all ranks of a short list of floats (every rank gets the result)."""
+    if world <= 1:
+        return list(values)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def job_value(tokens_per_rank, world, ms):
+    """Whole-job tokens/s: every rank processed `tokens_per_rank` in the (max-over-ranks) time `ms`."""
+    return world * tokens_per_rank / (ms * 1e-3)
+
+
 def oracle_sample_tokens_per_s(w, sample_T, verbose=False):
     """Time the fp64 oracle (as it stands) on a bounded sample: batch element 0, first sample_T tokens."""
     import numpy as np
@@ -210,10 +226,9 @@ def main():
     else:
         ms_e2e, h2d, d2h = run_e2e(args, torch, x, dy, grads, step, barrier, e0, e1)
 
-    if world > 1:
-        t = torch.tensor([ms, ms_e2e], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = t.tolist()
+    ms, ms_e2e = max_over_ranks([ms, ms_e2e if ms_e2e == ms_e2e else -1.0], dev, world)
+    if ms_e2e < 0:
+        ms_e2e = float("nan")
     report(args, B, w, world, rank, tokens, ms, ms_e2e, h2d, d2h, launches, phase, clocks)
     if world > 1:
         dist.destroy_process_group()
@@ -248,18 +263,26 @@ def report(args, B, w, world, rank, tokens, ms, ms_e2e, h2d, d2h, launches, phas
         bytes_per_token = w.d_model * (2 * e + 4 + 2 * e) + 2 * (2 * w.d_state * 4)   # see the design doc, adjoint main kernel
         k_ms = phase["adjoint_main"]
         achieved = bytes_per_token * tokens / (k_ms * 1e-3) / 1e9 if k_ms > 0 else None
+        # MUFU issue bound of the same kernel: >= 2 ex2 per (token, channel, state) in the chunk walk + 1/8 for the
+        # checkpoint fix-up + 1/16 for the sigmoid; 16 ex2 per clock per SM (measured), at the sampled SM clock
+        sm_mhz = (clocks or {}).get("sm_mhz") or 1965.0
+        ex2 = tokens * w.d_model * w.d_state * (2.0 + 1.0 / 8) + tokens * w.d_model
+        alu_peak = 16 * 148 * sm_mhz * 1e6
+        alu = {"kernel": "adjoint_main_kernel", "bound": "alu", "pipe": "MUFU.EX2", "achieved": ex2 / (k_ms * 1e-3) if k_ms > 0 else None,
+               "peak": alu_peak, "unit": "ex2/s", "frac": (ex2 / (k_ms * 1e-3) / alu_peak) if k_ms > 0 else None,
+               "sm_mhz": sm_mhz}
         traffic = None
         tpath = os.path.join(ROOT, "profiles", "traffic.json")
         if os.path.exists(tpath):
             traffic = json.load(open(tpath)).get(f"adjoint_main_kernel:{w.name}")
-        line = {"metric": METRIC, "value": world * tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        line = {"metric": METRIC, "value": job_value(tokens, world, ms), "unit": UNIT, "n_gpus": world,
                 "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": {"workload": w.name, "batch": w.batch, "seq_len": w.seqlen, "d_model": w.d_model,
                            "d_state": w.d_state, "tbar": w.tbar, "io": w.io, "layers": 1,
                            "parallelism": "replicas only" if world > 1 else "single GPU",
                            "l2": "inputs exceed L2 (x, dy, Delta: 0.8 GB per step)"},
-                "e2e": {"value": (world * tokens / (ms_e2e * 1e-3)) if ms_e2e == ms_e2e else None, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "e2e": {"value": job_value(tokens, world, ms_e2e) if ms_e2e == ms_e2e else None, "unit": UNIT, "h2d_bytes_per_step": h2d,
                         "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e if ms_e2e == ms_e2e else None},
                 "gpu_launches": launches,
                 "phases_ms": phase,
@@ -267,6 +290,7 @@ def report(args, B, w, world, rank, tokens, ms, ms_e2e, h2d, d2h, launches, phas
                              "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "traffic": traffic,
                              "peak_source": peak_src, "bytes_per_launch": bytes_per_token * tokens,
                              "launch_ms": k_ms},
+                "roofline_alu": alu,
                 "clocks": clocks}
         if world == 1 and not args.no_cpu_baseline:
             tps, dt, threads = oracle_sample_tokens_per_s(w, args.cpu_sample_tokens)
