@@ -104,7 +104,16 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-__device__ __forceinline__ float softplus_f(float u) { return fmaxf(u, 0.f) + log1pf(__expf(-fabsf(u))); }
+// softplus(u) = max(u,0) + log(1 + z), z = exp(-|u|) in (0,1]: two MUFU ops (ex2, lg2) and a short series
+// for small z, where forming 1 + z would lose z's low bits (relative error of the result < 3e-7)
+__device__ __forceinline__ float softplus_f(float u) {
+  const float z = ex2_approx(-fabsf(u) * LOG2E);
+  float l;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(l) : "f"(1.f + z));
+  const float big = l * LN2;
+  const float small = z * fmaf(z, fmaf(z, 1.f / 3.f, -0.5f), 1.f);   // z - z^2/2 + z^3/3
+  return fmaxf(u, 0.f) + (z < 0.0078125f ? small : big);
+}
 
 template <int AMAJ, int BMAJ, int EPI>
 __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,

@@ -680,7 +680,6 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
 #pragma unroll
         for (int jj = HALF - 1; jj >= 0; --jj) {
           const int j = k * HALF + jj;
-          __syncwarp();
           const float2 dv = lds_pair<float>(smd + St::D, jj, w.k);
           const float2 xv = lds_pair<IO>(smk + St::X, jj, w.k);
           const float2 gv = lds_pair<IO>(smk + St::G, jj, w.k);
