@@ -15,7 +15,7 @@
 namespace as {
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 64, STAGES = 3, UK = 16;
+constexpr int BM = 128, BN = 128, BK = 64, STAGES = 6, UK = 16, NTHREADS = 192;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int SMEM_DYN = STAGES * STAGE_BYTES + 1024;  // + slack for 1024-byte alignment
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
@@ -115,34 +115,41 @@ __device__ __forceinline__ float softplus_f(float u) {
   return fmaxf(u, 0.f) + (z < 0.0078125f ? small : big);
 }
 
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// Persistent, warp-specialised kernel: one CTA per SM walks tiles t = blockIdx.x, + gridDim.x, ...
+//   warp 0 (one lane): TMA producer over a STAGES-deep shared-memory ring that runs on across tiles
+//   warp 1 (one lane): tcgen05.mma issuer; the accumulator alternates between two 128-column TMEM buffers
+//   warps 2..5       : epilogue; drain buffer a while the issuer already fills buffer a^1 for the next tile
+// Tile order: n fastest, then m, then the K split, so concurrently running CTAs share A rows through L2.
 template <int AMAJ, int BMAJ, int EPI>
-__global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
-                                                      const __grid_constant__ CUtensorMap tmB, TcArgs a) {
+__global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
+                                                           const __grid_constant__ CUtensorMap tmB, TcArgs a) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[STAGES];
   __shared__ __align__(8) uint64_t empty_bar[STAGES];
-  __shared__ __align__(8) uint64_t tmem_full_bar;
+  __shared__ __align__(8) uint64_t tmem_full_bar[2];
+  __shared__ __align__(8) uint64_t tmem_empty_bar[2];
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
 
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int64_t m0 = (int64_t)blockIdx.x * BM;
-  const int n0 = blockIdx.y * BN;
+  const int mt = (int)((a.M + BM - 1) / BM), nt = (a.N + BN - 1) / BN;
+  const int ntiles = mt * nt * a.splitk;
   const int kper = (a.kblocks + a.splitk - 1) / a.splitk;
-  const int kb0 = blockIdx.z * kper;
-  const int kb1 = min(a.kblocks, kb0 + kper);
-  const int nkb = kb1 - kb0;
   volatile int* abortp = &abort_s;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-    mbar_init(&tmem_full_bar, 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full_bar[b], 1); mbar_init(&tmem_empty_bar[b], 4); }
     abort_s = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {   // TMEM allocation: BN fp32 accumulator columns
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(BN)
+  if (warp == 1) {   // TMEM allocation: two BN-column fp32 accumulators
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(2 * BN)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -151,115 +158,153 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CU
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = tmem_base_s;
 
-  if (nkb > 0) {
-    if (warp == 0 && lane == 0) {
+  auto decode = [&](int t, int64_t& m0, int& n0, int& kb0, int& nkb) {
+    const int in = t % nt, im = (t / nt) % mt, ik = t / (nt * mt);
+    m0 = (int64_t)im * BM; n0 = in * BN;
+    kb0 = ik * kper;
+    nkb = max(0, min(a.kblocks, kb0 + kper) - kb0);
+  };
+
+  if (warp == 0) {
+    if (lane == 0) {
       // ---------------- TMA producer ----------------
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
-      for (int i = 0; i < nkb; ++i) {
-        const int s = i % STAGES, round = i / STAGES;
-        if (round > 0 && !mbar_wait(&empty_bar[s], (round - 1) & 1, abortp)) { *abortp = 1; atomicExch(a.status, AS_ERR_TIMEOUT); break; }
-        uint8_t* sa = smem + s * STAGE_BYTES;
-        uint8_t* sb = sa + A_BYTES;
-        mbar_expect_tx(&full_bar[s], STAGE_BYTES);
-        const int k = (kb0 + i) * BK;
-        if (AMAJ == MAJ_K) {
-          tma_load_2d(sa, &tmA, k, (int)m0, &full_bar[s]);
-        } else {
-          tma_load_2d(sa, &tmA, (int)m0, k, &full_bar[s]);
-          tma_load_2d(sa + A_BYTES / 2, &tmA, (int)m0 + 64, k, &full_bar[s]);
-        }
-        if (BMAJ == MAJ_K) {
-          tma_load_2d(sb, &tmB, k, n0, &full_bar[s]);
-        } else {
-          tma_load_2d(sb, &tmB, n0, k, &full_bar[s]);
-          tma_load_2d(sb + B_BYTES / 2, &tmB, n0 + 64, k, &full_bar[s]);
+      int it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+        int64_t m0; int n0, kb0, nkb;
+        decode(t, m0, n0, kb0, nkb);
+        for (int i = 0; i < nkb; ++i, ++it) {
+          const int s = it % STAGES, round = it / STAGES;
+          if (round > 0 && !mbar_wait(&empty_bar[s], (round - 1) & 1, abortp)) { ok = false; break; }
+          uint8_t* sa = smem + s * STAGE_BYTES;
+          uint8_t* sb = sa + A_BYTES;
+          mbar_expect_tx(&full_bar[s], STAGE_BYTES);
+          const int k = (kb0 + i) * BK;
+          if (AMAJ == MAJ_K) {
+            tma_load_2d(sa, &tmA, k, (int)m0, &full_bar[s]);
+          } else {
+            tma_load_2d(sa, &tmA, (int)m0, k, &full_bar[s]);
+            tma_load_2d(sa + A_BYTES / 2, &tmA, (int)m0 + 64, k, &full_bar[s]);
+          }
+          if (BMAJ == MAJ_K) {
+            tma_load_2d(sb, &tmB, k, n0, &full_bar[s]);
+          } else {
+            tma_load_2d(sb, &tmB, n0, k, &full_bar[s]);
+            tma_load_2d(sb + B_BYTES / 2, &tmB, n0 + 64, k, &full_bar[s]);
+          }
         }
       }
-    } else if (warp == 1 && lane == 0) {
+      if (!ok) { *abortp = 1; atomicExch(a.status, AS_ERR_TIMEOUT); }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
       // ---------------- MMA issuer ----------------
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)AMAJ << 15) | ((uint32_t)BMAJ << 16) |
                              ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      int it = 0, ti = 0;
       bool ok = true;
-      for (int i = 0; i < nkb && ok; ++i) {
-        const int s = i % STAGES, round = i / STAGES;
-        if (!mbar_wait(&full_bar[s], round & 1, abortp)) { *abortp = 1; atomicExch(a.status, AS_ERR_TIMEOUT); ok = false; break; }
+      for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++ti) {
+        int64_t m0; int n0, kb0, nkb;
+        decode(t, m0, n0, kb0, nkb);
+        const int ab = ti & 1, around = ti >> 1;
+        if (around > 0 && !mbar_wait(&tmem_empty_bar[ab], (around - 1) & 1, abortp)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t sa = smem_u32(smem + s * STAGE_BYTES);
-        const uint32_t sb = sa + A_BYTES;
+        const uint32_t acc = tmem_base + (uint32_t)(ab * BN);
+        for (int i = 0; i < nkb; ++i, ++it) {
+          const int s = it % STAGES, round = it / STAGES;
+          if (!mbar_wait(&full_bar[s], round & 1, abortp)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t sa = smem_u32(smem + s * STAGE_BYTES);
+          const uint32_t sb = sa + A_BYTES;
 #pragma unroll
-        for (int k = 0; k < BK / UK; ++k) {
-          const uint64_t ad = (AMAJ == MAJ_K) ? make_desc(sa + k * UK * 2, 16, 1024)
-                                              : make_desc(sa + k * UK * 128, A_BYTES / 2, 1024);
-          const uint64_t bd = (BMAJ == MAJ_K) ? make_desc(sb + k * UK * 2, 16, 1024)
-                                              : make_desc(sb + k * UK * 128, B_BYTES / 2, 1024);
-          umma_bf16(tmem_base, ad, bd, idesc, (i > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < BK / UK; ++k) {
+            const uint64_t ad = (AMAJ == MAJ_K) ? make_desc(sa + k * UK * 2, 16, 1024)
+                                                : make_desc(sa + k * UK * 128, A_BYTES / 2, 1024);
+            const uint64_t bd = (BMAJ == MAJ_K) ? make_desc(sb + k * UK * 2, 16, 1024)
+                                                : make_desc(sb + k * UK * 128, B_BYTES / 2, 1024);
+            umma_bf16(acc, ad, bd, idesc, (i > 0 || k > 0) ? 1u : 0u);
+          }
+          umma_commit(&empty_bar[s]);   // frees the stage once these MMAs have read it
         }
-        umma_commit(&empty_bar[s]);   // frees the stage once these MMAs have read it
+        if (ok) umma_commit(&tmem_full_bar[ab]);   // accumulator of this tile complete
       }
-      umma_commit(&tmem_full_bar);    // accumulator complete
+      if (!ok) { *abortp = 1; atomicExch(a.status, AS_ERR_TIMEOUT); }
     }
-    // ---------------- epilogue: all four warps ----------------
-    __syncwarp();
-    const bool ready = mbar_wait(&tmem_full_bar, 0, abortp);
-    if (!ready) { *abortp = 1; if (lane == 0) atomicExch(a.status, AS_ERR_TIMEOUT); }
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (ready) {
-      const int64_t m = m0 + warp * 32 + lane;   // this thread's output row
+  } else {
+    // ---------------- epilogue warps ----------------
+    const int quarter = warp & 3;   // the TMEM lane quarter this warp may read
+    int ti = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++ti) {
+      int64_t m0; int n0, kb0, nkb;
+      decode(t, m0, n0, kb0, nkb);
+      const int ab = ti & 1, around = ti >> 1;
+      if (nkb > 0) {
+        if (!mbar_wait(&tmem_full_bar[ab], around & 1, abortp)) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int64_t m = m0 + quarter * 32 + lane;   // this thread's output row
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32), r);
-        const int nb = n0 + c * 32;
-        if (m >= a.M || nb >= a.N) continue;
-        if (EPI == TC_PROJ) {
-          if (nb < a.P) {
-            float4* dst = reinterpret_cast<float4*>(a.delta + m * a.P + nb);
-            const float4* b4 = reinterpret_cast<const float4*>(a.bias + nb);
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(ab * BN + c * 32), r);
+          const int nb = n0 + c * 32;
+          if (m >= a.M || nb >= a.N) continue;
+          if (EPI == TC_PROJ) {
+            if (nb < a.P) {
+              float4* dst = reinterpret_cast<float4*>(a.delta + m * a.P + nb);
+              const float4* b4 = reinterpret_cast<const float4*>(a.bias + nb);
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-              const float4 bv = __ldg(b4 + q);
-              dst[q] = make_float4(softplus_f(__uint_as_float(r[4 * q]) + bv.x), softplus_f(__uint_as_float(r[4 * q + 1]) + bv.y),
-                                   softplus_f(__uint_as_float(r[4 * q + 2]) + bv.z), softplus_f(__uint_as_float(r[4 * q + 3]) + bv.w));
+              for (int q = 0; q < 8; ++q) {
+                const float4 bv = __ldg(b4 + q);
+                dst[q] = make_float4(softplus_f(__uint_as_float(r[4 * q]) + bv.x), softplus_f(__uint_as_float(r[4 * q + 1]) + bv.y),
+                                     softplus_f(__uint_as_float(r[4 * q + 2]) + bv.z), softplus_f(__uint_as_float(r[4 * q + 3]) + bv.w));
+              }
+            } else {
+              float4* dst = reinterpret_cast<float4*>(a.bc + m * NBC + (nb - a.P));
+#pragma unroll
+              for (int q = 0; q < 8; ++q)
+                dst[q] = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]), __uint_as_float(r[4 * q + 2]),
+                                     __uint_as_float(r[4 * q + 3]));
             }
+          } else if (EPI == TC_DW) {
+            float* dst;
+            if (m < a.P) dst = a.dW_delta + m * a.P + nb;
+            else if (m < a.P + NS) dst = a.dW_B + (m - a.P) * a.P + nb;
+            else dst = a.dW_C + (m - a.P - NS) * a.P + nb;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) atomicAdd(dst + j, __uint_as_float(r[j]));
           } else {
-            float4* dst = reinterpret_cast<float4*>(a.bc + m * NBC + (nb - a.P));
+            const uint4* src = reinterpret_cast<const uint4*>(a.dxdir + m * a.P + nb);
+            uint4* dst = reinterpret_cast<uint4*>(a.dx + m * a.P + nb);
 #pragma unroll
-            for (int q = 0; q < 8; ++q)
-              dst[q] = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]), __uint_as_float(r[4 * q + 2]),
-                                   __uint_as_float(r[4 * q + 3]));
-          }
-        } else if (EPI == TC_DW) {
-          float* dst;
-          if (m < a.P) dst = a.dW_delta + m * a.P + nb;
-          else if (m < a.P + NS) dst = a.dW_B + (m - a.P) * a.P + nb;
-          else dst = a.dW_C + (m - a.P - NS) * a.P + nb;
+            for (int q = 0; q < 4; ++q) {
+              const uint4 sv = __ldg(src + q);
+              const __nv_bfloat162* s2 = reinterpret_cast<const __nv_bfloat162*>(&sv);
+              uint4 ov;
+              __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
 #pragma unroll
-          for (int j = 0; j < 32; ++j) atomicAdd(dst + j, __uint_as_float(r[j]));
-        } else {
-          const uint4* src = reinterpret_cast<const uint4*>(a.dxdir + m * a.P + nb);
-          uint4* dst = reinterpret_cast<uint4*>(a.dx + m * a.P + nb);
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const uint4 sv = __ldg(src + q);
-            const __nv_bfloat162* s2 = reinterpret_cast<const __nv_bfloat162*>(&sv);
-            uint4 ov;
-            __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const float2 f = __bfloat1622float2(s2[e]);
-              o2[e] = __floats2bfloat162_rn(f.x + __uint_as_float(r[8 * q + 2 * e]), f.y + __uint_as_float(r[8 * q + 2 * e + 1]));
+              for (int e = 0; e < 4; ++e) {
+                const float2 f = __bfloat1622float2(s2[e]);
+                o2[e] = __floats2bfloat162_rn(f.x + __uint_as_float(r[8 * q + 2 * e]), f.y + __uint_as_float(r[8 * q + 2 * e + 1]));
+              }
+              dst[q] = ov;
             }
-            dst[q] = ov;
           }
         }
+        // hand the accumulator buffer back to the issuer
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tmem_empty_bar[ab]);
       }
     }
+    if (!ok) { *abortp = 1; if (lane == 0) atomicExch(a.status, AS_ERR_TIMEOUT); }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (warp == 1) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(BN) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * BN) : "memory");
   }
 }
 
@@ -319,8 +364,9 @@ int launch_tc(const CUtensorMap& tmA, const CUtensorMap& tmB, const TcArgs& a, c
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN) != cudaSuccess) return 1;
     attr_set = true;
   }
-  dim3 grid((unsigned)((a.M + BM - 1) / BM), (unsigned)((a.N + BN - 1) / BN), (unsigned)a.splitk);
-  kern<<<grid, 128, SMEM_DYN, st>>>(tmA, tmB, a);
+  const int64_t ntiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN) * a.splitk;
+  const unsigned grid = (unsigned)(ntiles < 148 ? ntiles : 148);   // one persistent CTA per SM
+  kern<<<grid, NTHREADS, SMEM_DYN, st>>>(tmA, tmB, a);
   count_launch();
   return (int)cudaGetLastError();
 }
@@ -362,10 +408,11 @@ int tc_weight_grads(const Plan& pl, const void* x, const as_grads_t* out, char* 
   TcArgs a{};
   a.M = NW; a.N = P; a.kblocks = (int)((M + BK - 1) / BK); a.P = P;
   const int tiles = ((NW + BM - 1) / BM) * ((P + BN - 1) / BN);
-  int sk = (148 * 2 + tiles - 1) / tiles;
+  int sk = (148 * 2) / tiles;   // about two tiles per persistent CTA
   if (sk > a.kblocks) sk = a.kblocks;
   if (sk < 1) sk = 1;
-  a.splitk = sk;
+  const int kper = (a.kblocks + sk - 1) / sk;
+  a.splitk = (a.kblocks + kper - 1) / kper;   // no empty split: every tile has at least one K block
   a.dW_delta = out->dW_delta; a.dW_B = out->dW_B; a.dW_C = out->dW_C;
   a.status = (int*)(ws + pl.off_status);
   return launch_tc<MAJ_MN, MAJ_MN, TC_DW>(tmA, tmB, a, st);
