@@ -155,6 +155,7 @@ struct Stage {
   static constexpr int BYTES = BC2 + (WIN ? CK * NBC * 4 : 0);
 };
 constexpr int NSTAGE = 3;        // ascending kernels
+constexpr int WRED_Q = 32 * 4 + 8;   // floats per quarter-block of the per-warp reduction scratch (512 B + 32 B skew)
 constexpr int HALF = CK / 2;       // tokens per unrolled loop body of the main adjoint kernel
 constexpr int NSTAGE_MAIN = 2;   // main adjoint kernel: a chunk takes thousands of cycles, one chunk of lookahead suffices
 
@@ -512,7 +513,8 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   using St = Stage<ESZ, true, true, WIN>;
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[NSTAGE_MAIN];
-  __shared__ float red[2][CH / 32][CK][NBC];
+  __shared__ float red[2][CK][NBC];                 // per-token [dB | dC] sums of the CTA, two chunks in flight
+  __shared__ __align__(16) float wred[CH / 32][4 * WRED_Q];   // per-warp scratch of the channel reduction
   __shared__ ulonglong2 hst_s[4][CH];
   uint8_t* smem = smem_raw + ((128u - (smem_u32(smem_raw) & 127u)) & 127u);   // stays a shared-space pointer
 
@@ -540,6 +542,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     for (int i = 0; i < NSTAGE_MAIN; ++i) mbar_init(&full_bar[i], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  for (int e = w.tid; e < 2 * CK * NBC; e += CH) (&red[0][0][0])[e] = 0.f;
   __syncthreads();
   const uint32_t tx_base = (uint32_t)(CK * CH * ESZ * 2 + CK * CH * 4 + CK * NBC * 4 + TILE_FLOATS * 4 + ncs * 4 +
                                       (WIN ? CK * CH * ESZ + CK * CH * 4 : 0));
@@ -764,23 +767,25 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
               st_io<IO>(dxdir + row * P, d * sv);
             }
           }
-          // transposing reduction over the 16 lanes of equal parity: afterwards this lane holds the warp total of
-          // value (lane >> 1): values 0..7 = dB[8*half + .], 8..15 = dC[8*half + .]
-          float v[16];
+          // sum over the warp's 16 channel pairs: every lane parks its 16 partials (dB[8*half+0..7], dC[8*half+0..7])
+          // in shared memory, then lane l adds up value (l >> 1) over the 16 lanes of its parity.  Quarter-blocks
+          // of 4 values are 544 bytes apart so that both the 16-byte stores and the 4-byte loads are conflict-free.
+          {
+            float* wr = wred[warp];
+            __syncwarp();   // the previous token's loads from wr are done
 #pragma unroll
-          for (int m = 0; m < 4; ++m) { upk(vB[m], v[2 * m], v[2 * m + 1]); upk(vC[m], v[8 + 2 * m], v[8 + 2 * m + 1]); }
-#pragma unroll
-          for (int off = 16, cnt = 8; cnt >= 1; off >>= 1, cnt >>= 1) {
-            const bool up = (lane & off) != 0;
-#pragma unroll
-            for (int kk = 0; kk < cnt; ++kk) {
-              const float send = up ? v[kk] : v[kk + cnt];
-              const float keep = up ? v[kk + cnt] : v[kk];
-              v[kk] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+            for (int m = 0; m < 4; ++m) {
+              const u64* src = (m < 2) ? &vB[2 * m] : &vC[2 * (m - 2)];
+              *reinterpret_cast<ulonglong2*>(wr + m * WRED_Q + lane * 4) = make_ulonglong2(src[0], src[1]);
             }
+            __syncwarp();
+            const int vi = lane >> 1;
+            const float* rd = wr + (vi >> 2) * WRED_Q + (lane & 1) * 4 + (vi & 3);
+            float tot = 0.f;
+#pragma unroll
+            for (int i2 = 0; i2 < 16; ++i2) tot += rd[i2 * 8];
+            atomicAdd(&red[rb][j][(vi & 8) * 2 + 8 * w.half + (vi & 7)], tot);
           }
-          const int vi = lane >> 1;
-          red[rb][warp][j][(vi & 8) * 2 + 8 * w.half + (vi & 7)] = v[0];
         }
       }
     }
@@ -791,12 +796,11 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
       return;
     }
     if (w.tid == 0 && i + NSTAGE_MAIN < nchunk) issue(i + NSTAGE_MAIN);
-    for (int e = w.tid; e < nt * NBC; e += CH) {
+    for (int e = w.tid; e < CK * NBC; e += CH) {
       const int j = e / NBC, q = e % NBC;
-      float sum = 0.f;
-#pragma unroll
-      for (int wq = 0; wq < CH / 32; ++wq) sum += red[rb][wq][j][q];
-      atomicAdd(dbc + ((int64_t)b * T + tc + j) * NBC + q, sum);
+      const float sum = red[rb][j][q];
+      red[rb][j][q] = 0.f;   // ready for the chunk after next
+      if (j < nt) atomicAdd(dbc + ((int64_t)b * T + tc + j) * NBC + q, sum);
     }
   }
   if (w.act) {
