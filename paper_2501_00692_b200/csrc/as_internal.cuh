@@ -17,7 +17,10 @@ inline void count_launch(int n = 1) { g_launches.fetch_add(n); }
 
 constexpr int NS = 16;        // d_state handled by the scan kernels
 constexpr int CK = 8;         // tokens per checkpoint chunk (h of one chunk lives in registers)
-constexpr int CH = 128;       // channels per CTA of the scan kernels
+constexpr int NCH = 2;        // channels per thread of the scan kernels (1 or 2)
+constexpr int NTHR = 128;     // threads per CTA of the scan kernels; two threads share a channel set, 8 states each
+constexpr int CH = NTHR / 2 * NCH;   // channels per CTA
+constexpr int NU = 4 * NCH;   // packed state pairs (f32x2) a thread owns
 constexpr int TILE_FLOATS = CH * NS;   // one (channel tile, all states) block of a per-segment / per-chunk array
 constexpr int NBC = 2 * NS;   // per-token row of [B_t | C_t] (and of [dB_t | dC_t])
 constexpr float LOG2E = 1.4426950408889634f;
@@ -45,7 +48,7 @@ __device__ __forceinline__ float ex2_approx(float x) {
 // Time is cut into S segments of L tokens (L a multiple of CK); a CTA owns (segment, batch element,
 // CH channels).  Per-(segment, channel, state) and per-(chunk, channel, state) arrays are stored as
 // blocks of TILE_FLOATS floats per channel tile, in the order the owning thread keeps them in registers
-// (float4 q of thread tid at float offset (q*CH + tid)*4), so one bulk copy moves a CTA's block and
+// (float4 q of thread tid at float offset (q*NTHR + tid)*4), so one bulk copy moves a CTA's block and
 // every thread's access is a contiguous 16 bytes.
 struct Plan {
   int B, P;

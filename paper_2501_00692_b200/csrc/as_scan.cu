@@ -31,8 +31,10 @@ int make_plan(const as_shape_t* sh, int64_t tbar, Plan* pl) {
   p.tiles = (p.P + CH - 1) / CH;
   p.bw = p.P < CH ? p.P : CH;
   const int64_t ctas = (int64_t)p.tiles * p.B;
-  const int64_t target = 148 * 2 * 4;
-  int64_t s_target = (target + ctas - 1) / ctas;
+  // two full waves of the main kernel's resident CTAs (148 SMs x CTAs per SM), never more than that
+  const int64_t slots = 148 * (NCH == 2 ? 3 : 4);
+  int64_t s_target = (2 * slots) / ctas;
+  if (s_target < 1) s_target = 1;
   int64_t L = (p.T + s_target - 1) / s_target;
   L = (L + CK - 1) / CK * CK;
   if (L < 64) L = 64;
@@ -156,60 +158,90 @@ struct Stage {
 };
 constexpr int NSTAGE = 3;        // ascending kernels
 constexpr int WRED_Q = 32 * 4 + 8;   // floats per quarter-block of the per-warp reduction scratch (512 B + 32 B skew)
+constexpr int MAIN_CTAS = NCH == 2 ? 3 : 4;   // resident CTAs per SM the main kernel is compiled for
 constexpr int HALF = CK / 2;       // tokens per unrolled loop body of the main adjoint kernel
 constexpr int NSTAGE_MAIN = 2;   // main adjoint kernel: a chunk takes thousands of cycles, one chunk of lookahead suffices
 
-template <typename IO> __device__ __forceinline__ float2 lds_pair(const uint8_t* tile, int j, int k);
-template <> __device__ __forceinline__ float2 lds_pair<float>(const uint8_t* tile, int j, int k) {
-  return *reinterpret_cast<const float2*>(tile + (j * CH + 2 * k) * 4);
+// per-thread values of its NCH channels
+struct ChV { float v[NCH]; };
+__device__ __forceinline__ ChV ch_zero() { ChV r; for (int c = 0; c < NCH; ++c) r.v[c] = 0.f; return r; }
+
+// row j of a staged [CK x CH] tile, channels NCH*k .. NCH*k + NCH-1
+template <typename IO> __device__ __forceinline__ ChV lds_ch(const uint8_t* tile, int j, int k);
+template <> __device__ __forceinline__ ChV lds_ch<float>(const uint8_t* tile, int j, int k) {
+  ChV r;
+  if (NCH == 2) {
+    const float2 t = *reinterpret_cast<const float2*>(tile + (j * CH + 2 * k) * 4);
+    r.v[0] = t.x; r.v[NCH - 1] = t.y;
+  } else {
+    r.v[0] = *reinterpret_cast<const float*>(tile + (j * CH + k) * 4);
+  }
+  return r;
 }
-template <> __device__ __forceinline__ float2 lds_pair<__nv_bfloat16>(const uint8_t* tile, int j, int k) {
-  const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(tile + (j * CH + 2 * k) * 2);
-  return __bfloat1622float2(v);
+template <> __device__ __forceinline__ ChV lds_ch<__nv_bfloat16>(const uint8_t* tile, int j, int k) {
+  ChV r;
+  if (NCH == 2) {
+    const float2 t = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(tile + (j * CH + 2 * k) * 2));
+    r.v[0] = t.x; r.v[NCH - 1] = t.y;
+  } else {
+    r.v[0] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(tile + (j * CH + k) * 2));
+  }
+  return r;
+}
+// NCH consecutive floats of a global per-channel array
+__device__ __forceinline__ ChV ldg_ch(const float* p) {
+  ChV r;
+#pragma unroll
+  for (int c = 0; c < NCH; ++c) r.v[c] = __ldg(p + c);
+  return r;
+}
+__device__ __forceinline__ void stg_ch(float* p, const float (&v)[NCH]) {
+#pragma unroll
+  for (int c = 0; c < NCH; ++c) p[c] = v[c];
 }
 
 struct Who {          // what this thread owns
   int tid, k, half;   // pair index, state half
-  int pa;             // first channel (second is pa + 1)
-  bool act;           // channels exist (P is even, so both or neither)
+  int pa;             // first of its NCH channels
+  bool act;           // the channels exist (P is a multiple of 8, so all or none)
 };
 __device__ __forceinline__ Who who(int tile, int P) {
   Who w;
   w.tid = threadIdx.x; w.k = w.tid >> 1; w.half = w.tid & 1;
-  w.pa = tile * CH + 2 * w.k;
+  w.pa = tile * CH + NCH * w.k;
   w.act = w.pa < P;
   return w;
 }
 // A2[u] = -exp(A_log) * log2(e) for unit u = ch*4 + m  ->  states (8*half + 2m, +1) of channel pa + ch
-__device__ __forceinline__ void load_A2(const float* A_log, const Who& w, u64 (&A2)[8]) {
+__device__ __forceinline__ void load_A2(const float* A_log, const Who& w, u64 (&A2)[NU]) {
 #pragma unroll
-  for (int u = 0; u < 8; ++u) {
+  for (int u = 0; u < NU; ++u) {
     float2 v = make_float2(0.f, 0.f);
     if (w.act) v = __ldg(reinterpret_cast<const float2*>(A_log + (int64_t)(w.pa + u / 4) * NS + 8 * w.half + 2 * (u % 4)));
     A2[u] = pk(-__expf(v.x) * LOG2E, -__expf(v.y) * LOG2E);
   }
 }
 // 16 values of this thread inside a 2048-float tile block: float4 q of thread tid at (q*128 + tid)
-__device__ __forceinline__ void load_block(const float* blk, int tid, u64 (&v)[8]) {
+__device__ __forceinline__ void load_block(const float* blk, int tid, u64 (&v)[NU]) {
   const ulonglong2* b2 = reinterpret_cast<const ulonglong2*>(blk);
 #pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const ulonglong2 t = b2[q * CH + tid];
+  for (int q = 0; q < 2 * NCH; ++q) {
+    const ulonglong2 t = b2[q * NTHR + tid];
     v[2 * q] = t.x; v[2 * q + 1] = t.y;
   }
 }
-__device__ __forceinline__ void load_block_g(const float* blk, int tid, u64 (&v)[8]) {
+__device__ __forceinline__ void load_block_g(const float* blk, int tid, u64 (&v)[NU]) {
   const ulonglong2* b2 = reinterpret_cast<const ulonglong2*>(blk);
 #pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const ulonglong2 t = __ldg(b2 + q * CH + tid);
+  for (int q = 0; q < 2 * NCH; ++q) {
+    const ulonglong2 t = __ldg(b2 + q * NTHR + tid);
     v[2 * q] = t.x; v[2 * q + 1] = t.y;
   }
 }
-__device__ __forceinline__ void store_block(float* blk, int tid, const u64 (&v)[8]) {
+__device__ __forceinline__ void store_block(float* blk, int tid, const u64 (&v)[NU]) {
   ulonglong2* b2 = reinterpret_cast<ulonglong2*>(blk);
 #pragma unroll
-  for (int q = 0; q < 4; ++q) b2[q * CH + tid] = make_ulonglong2(v[2 * q], v[2 * q + 1]);
+  for (int q = 0; q < 2 * NCH; ++q) b2[q * NTHR + tid] = make_ulonglong2(v[2 * q], v[2 * q + 1]);
 }
 
 // sigmoid(u) from Delta = softplus(u): 1 - exp(-Delta), without cancellation for small Delta
@@ -240,11 +272,11 @@ enum { PRE_FWD = 0, PRE_ADJ = 1, PRE_Y = 2 };
 __device__ __forceinline__ void zero_rows(uint8_t* tile, int row_bytes, int nt, int tid) {
   uint4* p = reinterpret_cast<uint4*>(tile + nt * row_bytes);
   const int n16 = (CK - nt) * row_bytes / 16;
-  for (int i = tid; i < n16; i += CH) p[i] = make_uint4(0u, 0u, 0u, 0u);
+  for (int i = tid; i < n16; i += NTHR) p[i] = make_uint4(0u, 0u, 0u, 0u);
 }
 
 template <typename IO, int MODE>
-__global__ void __launch_bounds__(CH) ascend_kernel(const __grid_constant__ CUtensorMap tmX,
+__global__ void __launch_bounds__(NTHR) ascend_kernel(const __grid_constant__ CUtensorMap tmX,
                                                     const __grid_constant__ CUtensorMap tmD,
                                                     const __grid_constant__ CUtensorMap tmG, Plan pl,
                                                     const float* __restrict__ A_log, char* __restrict__ ws,
@@ -284,18 +316,20 @@ __global__ void __launch_bounds__(CH) ascend_kernel(const __grid_constant__ CUte
   if (w.tid == 0)
     for (int c = 0; c < NSTAGE && c < nchunk; ++c) issue(c);
 
-  u64 A2[8], h[8], Pr[8], acc[8], snap[8];
+  u64 A2[NU], h[NU], Pr[NU], acc[NU], snap[NU];
   load_A2(A_log, w, A2);
   const int64_t sb = ((int64_t)b * pl.S + s) * pl.tiles + tile;
   if (MODE == PRE_Y) {
     load_block_g(reinterpret_cast<const float*>(ws + pl.off_hstart) + sb * TILE_FLOATS, w.tid, h);
   } else {
 #pragma unroll
-    for (int u = 0; u < 8; ++u) h[u] = 0ull;
+    for (int u = 0; u < NU; ++u) h[u] = 0ull;
   }
 #pragma unroll
-  for (int u = 0; u < 8; ++u) { Pr[u] = pk(1.f, 1.f); acc[u] = 0ull; snap[u] = 0ull; }
-  float cum[2] = {0.f, 0.f}, partd[2] = {0.f, 0.f};
+  for (int u = 0; u < NU; ++u) { Pr[u] = pk(1.f, 1.f); acc[u] = 0ull; snap[u] = 0ull; }
+  float cum[NCH], partd[NCH];
+#pragma unroll
+  for (int c = 0; c < NCH; ++c) { cum[c] = 0.f; partd[c] = 0.f; }
 
   for (int c = 0; c < nchunk; ++c) {
     const int st = c % NSTAGE;
@@ -308,7 +342,7 @@ __global__ void __launch_bounds__(CH) ascend_kernel(const __grid_constant__ CUte
       const int64_t cc = ((int64_t)b * pl.NC + tc / CK);
       store_block(reinterpret_cast<float*>(ws + pl.off_ckpt) + (cc * pl.tiles + tile) * TILE_FLOATS, w.tid, h);
       if (w.half == 0 && w.act)
-        *reinterpret_cast<float2*>(reinterpret_cast<float*>(ws + pl.off_cs) + cc * P + w.pa) = make_float2(cum[0], cum[1]);
+        stg_ch(reinterpret_cast<float*>(ws + pl.off_cs) + cc * P + w.pa, cum);
     }
     if (nt < CK) {   // only the last chunk of a sequence
       if (ok) {
@@ -322,10 +356,10 @@ __global__ void __launch_bounds__(CH) ascend_kernel(const __grid_constant__ CUte
 #pragma unroll
       for (int j = 0; j < CK; ++j) {
         // channels past P read the zero fill of the TMA box: Delta = x = g = 0 keeps their slots at zero
-        const float2 dv = lds_pair<float>(sm + St::D, j, w.k);
-        const float2 xv = lds_pair<IO>(sm + St::X, j, w.k);
-        float2 gv = make_float2(0.f, 0.f);
-        if (MU) gv = lds_pair<IO>(sm + St::G, j, w.k);
+        const ChV dv = lds_ch<float>(sm + St::D, j, w.k);
+        const ChV xv = lds_ch<IO>(sm + St::X, j, w.k);
+        ChV gv = ch_zero();
+        if (MU) gv = lds_ch<IO>(sm + St::G, j, w.k);
         const float* brow = reinterpret_cast<const float*>(sm + St::BC) + j * NBC + 8 * w.half;
         const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
         const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
@@ -336,13 +370,12 @@ __global__ void __launch_bounds__(CH) ascend_kernel(const __grid_constant__ CUte
           const ulonglong2 c23 = *reinterpret_cast<const ulonglong2*>(brow + NS + 4);
           Cp[0] = c01.x; Cp[1] = c01.y; Cp[2] = c23.x; Cp[3] = c23.y;
         }
-        const float dd[2] = {dv.x, dv.y};
-        const float dxs[2] = {dv.x * xv.x, dv.y * xv.y};
-        const float gs[2] = {gv.x, gv.y};
-        float yv[2] = {0.f, 0.f};
+        float yv[NCH];
 #pragma unroll
-        for (int ch = 0; ch < 2; ++ch) {
-          const u64 d2 = pk(dd[ch], dd[ch]), dx2 = pk(dxs[ch], dxs[ch]), g2 = pk(gs[ch], gs[ch]);
+        for (int ch = 0; ch < NCH; ++ch) {
+          const float ddc = dv.v[ch], dxc = dv.v[ch] * xv.v[ch], gc = gv.v[ch];
+          const u64 d2 = pk(ddc, ddc), dx2 = pk(dxc, dxc), g2 = pk(gc, gc);
+          yv[ch] = 0.f;
           u64 yacc = 0ull;
 #pragma unroll
           for (int m = 0; m < 4; ++m) {
@@ -356,17 +389,21 @@ __global__ void __launch_bounds__(CH) ascend_kernel(const __grid_constant__ CUte
             if (MODE == PRE_Y) yacc = fma2(Cp[m], h[u], yacc);
           }
           if (MODE == PRE_Y) yv[ch] = hsum(yacc);
-          cum[ch] += dd[ch];
+          cum[ch] += ddc;
         }
         if (MODE == PRE_Y) {
-          yv[0] += __shfl_xor_sync(0xffffffffu, yv[0], 1);
-          yv[1] += __shfl_xor_sync(0xffffffffu, yv[1], 1);
-          if (w.act && j < nt) st_io<IO>(y + ((int64_t)b * pl.T + tc + j) * P + w.pa + w.half, w.half ? yv[1] : yv[0]);
+#pragma unroll
+          for (int ch = 0; ch < NCH; ++ch) yv[ch] += __shfl_xor_sync(0xffffffffu, yv[ch], 1);
+          // the two lanes of a pair hold the same sums: lane `half` writes channel `half` (one channel per thread: lane 0)
+          const int chf = NCH == 2 ? w.half : 0;
+          if (w.act && j < nt && (NCH == 2 || w.half == 0))
+            st_io<IO>(y + ((int64_t)b * pl.T + tc + j) * P + w.pa + chf, yv[chf]);
         }
         if (MU && j == jr) {
-          partd[0] = cum[0]; partd[1] = cum[1];
 #pragma unroll
-          for (int u = 0; u < 8; ++u) snap[u] = acc[u];
+          for (int c = 0; c < NCH; ++c) partd[c] = cum[c];
+#pragma unroll
+          for (int u = 0; u < NU; ++u) snap[u] = acc[u];
         }
       }
     }
@@ -379,15 +416,16 @@ __global__ void __launch_bounds__(CH) ascend_kernel(const __grid_constant__ CUte
   }
   if (MODE == PRE_Y) return;
   if (MU && (t1 - t0) < pl.r) {   // ragged last segment shorter than r tokens: the snapshot is the whole segment
-    partd[0] = cum[0]; partd[1] = cum[1];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) snap[u] = acc[u];
+    for (int c = 0; c < NCH; ++c) partd[c] = cum[c];
+#pragma unroll
+    for (int u = 0; u < NU; ++u) snap[u] = acc[u];
   }
   store_block(reinterpret_cast<float*>(ws + pl.off_hend) + sb * TILE_FLOATS, w.tid, h);
   const int64_t sp = ((int64_t)b * pl.S + s) * P + w.pa;
   if (w.half == 0 && w.act) {
-    *reinterpret_cast<float2*>(reinterpret_cast<float*>(ws + pl.off_segd) + sp) = make_float2(cum[0], cum[1]);
-    if (MU) *reinterpret_cast<float2*>(reinterpret_cast<float*>(ws + pl.off_partd) + sp) = make_float2(partd[0], partd[1]);
+    stg_ch(reinterpret_cast<float*>(ws + pl.off_segd) + sp, cum);
+    if (MU) stg_ch(reinterpret_cast<float*>(ws + pl.off_partd) + sp, partd);
   }
   if (MU) {
     store_block(reinterpret_cast<float*>(ws + pl.off_muloc) + sb * TILE_FLOATS, w.tid, acc);
@@ -399,26 +437,26 @@ __global__ void __launch_bounds__(CH) ascend_kernel(const __grid_constant__ CUte
 // carries across segments.  Thread (b, tile, tid) owns the same 16 (channel, state) slots as in the scans.
 // ------------------------------------------------------------------------------------------------
 // hstart[s]: true state entering segment s (sequential in s).
-__global__ void __launch_bounds__(CH) fixup_h_kernel(Plan pl, const float* __restrict__ A_log, char* __restrict__ ws) {
+__global__ void __launch_bounds__(NTHR) fixup_h_kernel(Plan pl, const float* __restrict__ A_log, char* __restrict__ ws) {
   const int tile = blockIdx.x, b = blockIdx.y;
   const Who w = who(tile, pl.P);
-  u64 A2[8], hs[8];
+  u64 A2[NU], hs[NU];
   load_A2(A_log, w, A2);
 #pragma unroll
-  for (int u = 0; u < 8; ++u) hs[u] = 0ull;
+  for (int u = 0; u < NU; ++u) hs[u] = 0ull;
   const float* hend = reinterpret_cast<const float*>(ws + pl.off_hend);
   const float* segd = reinterpret_cast<const float*>(ws + pl.off_segd);
   float* hstart = reinterpret_cast<float*>(ws + pl.off_hstart);
   constexpr int UN = 4;
   for (int s0 = 0; s0 < pl.S; s0 += UN) {
-    u64 he[UN][8];
-    float2 sd[UN];
+    u64 he[UN][NU];
+    ChV sd[UN];
 #pragma unroll
     for (int i = 0; i < UN; ++i) {
       const int s = min(s0 + i, pl.S - 1);
       const int64_t sb = ((int64_t)b * pl.S + s) * pl.tiles + tile;
       load_block_g(hend + sb * TILE_FLOATS, w.tid, he[i]);
-      sd[i] = w.act ? __ldg(reinterpret_cast<const float2*>(segd + ((int64_t)b * pl.S + s) * pl.P + w.pa)) : make_float2(0.f, 0.f);
+      sd[i] = w.act ? ldg_ch(segd + ((int64_t)b * pl.S + s) * pl.P + w.pa) : ch_zero();
     }
 #pragma unroll
     for (int i = 0; i < UN; ++i) {
@@ -426,9 +464,11 @@ __global__ void __launch_bounds__(CH) fixup_h_kernel(Plan pl, const float* __res
       if (s < pl.S) {
         const int64_t sb = ((int64_t)b * pl.S + s) * pl.tiles + tile;
         store_block(hstart + sb * TILE_FLOATS, w.tid, hs);
-        const u64 d2[2] = {pk(sd[i].x, sd[i].x), pk(sd[i].y, sd[i].y)};
+        u64 d2[NCH];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) hs[u] = fma2(ex2_2(mul2(d2[u / 4], A2[u])), hs[u], he[i][u]);
+        for (int c = 0; c < NCH; ++c) d2[c] = pk(sd[i].v[c], sd[i].v[c]);
+#pragma unroll
+        for (int u = 0; u < NU; ++u) hs[u] = fma2(ex2_2(mul2(d2[u / 4], A2[u])), hs[u], he[i][u]);
       }
     }
   }
@@ -439,11 +479,11 @@ __global__ void __launch_bounds__(CH) fixup_h_kernel(Plan pl, const float* __res
 //   mu_loc[s+1] + D[s+1] (mu_loc[s+2] + ... + D[s+m] mu_part[s+m+1]),   D[s'] = exp(A * sum of Delta over s'),
 // i.e. m whole segments plus the first r tokens of the next one (all later segments in the full form).
 // swin[s]: sum of Delta over the Tbar tokens after e (fp64), for the window-exit factor.
-__global__ void __launch_bounds__(CH) fixup_mu_kernel(Plan pl, const float* __restrict__ A_log, char* __restrict__ ws) {
+__global__ void __launch_bounds__(NTHR) fixup_mu_kernel(Plan pl, const float* __restrict__ A_log, char* __restrict__ ws) {
   const int tile = blockIdx.x, b = blockIdx.z;
   const int P = pl.P, S = pl.S;
   const Who w = who(tile, P);
-  u64 A2[8];
+  u64 A2[NU];
   load_A2(A_log, w, A2);
   const float* muloc = reinterpret_cast<const float*>(ws + pl.off_muloc);
   const float* mupart = reinterpret_cast<const float*>(ws + pl.off_mupart);
@@ -452,22 +492,24 @@ __global__ void __launch_bounds__(CH) fixup_mu_kernel(Plan pl, const float* __re
   float* carry = reinterpret_cast<float*>(ws + pl.off_carry);
   double* swin = reinterpret_cast<double*>(ws + pl.off_swin);
   auto blk = [&](int s) -> int64_t { return (((int64_t)b * S + s) * pl.tiles + tile) * TILE_FLOATS; };
-  auto ld2 = [&](const float* arr, int s) -> float2 {
-    return (w.act && s < S) ? __ldg(reinterpret_cast<const float2*>(arr + ((int64_t)b * S + s) * P + w.pa)) : make_float2(0.f, 0.f);
+  auto ld2 = [&](const float* arr, int s) -> ChV {
+    return (w.act && s < S) ? ldg_ch(arr + ((int64_t)b * S + s) * P + w.pa) : ch_zero();
   };
-  auto step = [&](int sg, u64 (&val)[8]) {   // val = mu_loc[sg] + D[sg] * val
-    const float2 sd = ld2(segd, sg);
-    const u64 d2[2] = {pk(sd.x, sd.x), pk(sd.y, sd.y)};
-    u64 ml[8];
+  auto step = [&](int sg, u64 (&val)[NU]) {   // val = mu_loc[sg] + D[sg] * val
+    const ChV sd = ld2(segd, sg);
+    u64 d2[NCH];
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) d2[c] = pk(sd.v[c], sd.v[c]);
+    u64 ml[NU];
     load_block_g(muloc + blk(sg), w.tid, ml);
 #pragma unroll
-    for (int u = 0; u < 8; ++u) val[u] = fma2(ex2_2(mul2(d2[u / 4], A2[u])), val[u], ml[u]);
+    for (int u = 0; u < NU; ++u) val[u] = fma2(ex2_2(mul2(d2[u / 4], A2[u])), val[u], ml[u]);
   };
   if (pl.full) {
     if (blockIdx.y != 0) return;
-    u64 val[8];
+    u64 val[NU];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) val[u] = 0ull;
+    for (int u = 0; u < NU; ++u) val[u] = 0ull;
     for (int s = S - 1; s >= 0; --s) {
       store_block(carry + blk(s), w.tid, val);
       step(s, val);
@@ -475,9 +517,9 @@ __global__ void __launch_bounds__(CH) fixup_mu_kernel(Plan pl, const float* __re
   } else {
     const int s = blockIdx.y;
     const int s1 = s + 1;
-    u64 val[8];
+    u64 val[NU];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) val[u] = 0ull;
+    for (int u = 0; u < NU; ++u) val[u] = 0ull;
     if (s1 + pl.m < S) load_block_g(mupart + blk(s1 + pl.m), w.tid, val);
     for (int k = pl.m - 1; k >= 0; --k) {
       const int sg = s1 + k;
@@ -485,12 +527,18 @@ __global__ void __launch_bounds__(CH) fixup_mu_kernel(Plan pl, const float* __re
     }
     store_block(carry + blk(s), w.tid, val);
     if (w.half == 0 && w.act) {
-      double sw0 = 0.0, sw1 = 0.0;
-      for (int k = 1; k <= pl.m; ++k) { const float2 v = ld2(segd, s + k); sw0 += (double)v.x; sw1 += (double)v.y; }
-      const float2 pv = ld2(partd, s + pl.m + 1);
-      sw0 += (double)pv.x; sw1 += (double)pv.y;
+      double swv[NCH];
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) swv[c] = 0.0;
+      for (int k = 1; k <= pl.m; ++k) {
+        const ChV v = ld2(segd, s + k);
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) swv[c] += (double)v.v[c];
+      }
+      const ChV pv = ld2(partd, s + pl.m + 1);
       double* dst = swin + ((int64_t)b * S + s) * P + w.pa;
-      dst[0] = sw0; dst[1] = sw1;
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) dst[c] = swv[c] + (double)pv.v[c];
     }
   }
 }
@@ -504,7 +552,7 @@ __global__ void __launch_bounds__(CH) fixup_mu_kernel(Plan pl, const float* __re
 //   and evaluating the per-token VJPs.
 // ------------------------------------------------------------------------------------------------
 template <typename IO, bool FULL>
-__global__ void __launch_bounds__(CH, 3)
+__global__ void __launch_bounds__(NTHR, MAIN_CTAS)
 adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmD,
                     const __grid_constant__ CUtensorMap tmG, Plan pl, const float* __restrict__ A_log,
                     char* __restrict__ ws, float* __restrict__ dA_log, float* __restrict__ db_delta) {
@@ -514,8 +562,8 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[NSTAGE_MAIN];
   __shared__ float red[2][CK][NBC];                 // per-token [dB | dC] sums of the CTA, two chunks in flight
-  __shared__ __align__(16) float wred[CH / 32][4 * WRED_Q];   // per-warp scratch of the channel reduction
-  __shared__ ulonglong2 hst_s[4][CH];
+  __shared__ __align__(16) float wred[NTHR / 32][4 * WRED_Q];   // per-warp scratch of the channel reduction
+  __shared__ ulonglong2 hst_s[2 * NCH][NTHR];
   uint8_t* smem = smem_raw + ((128u - (smem_u32(smem_raw) & 127u)) & 127u);   // stays a shared-space pointer
 
   const int tile = blockIdx.x, s = blockIdx.y, b = blockIdx.z;
@@ -534,7 +582,11 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   const int ncs = min(CH, P - tile * CH);   // channels of this tile that exist
   const int64_t BT = (int64_t)pl.B * T;
   const int du_ld = pl.du_ld;
-  const int pmine = w.pa + w.half;   // the channel whose per-token outputs this lane finalises
+  // the two lanes of a pair end up with the same per-channel sums: with two channels per thread lane `half`
+  // finalises channel `half`, with one channel per thread lane 0 does
+  const int chf = NCH == 2 ? w.half : 0;
+  const bool fin = w.act && (NCH == 2 || w.half == 0);
+  const int pmine = w.pa + chf;
   IO* du = reinterpret_cast<IO*>(ws + pl.off_du) + pmine;
   IO* dxdir = reinterpret_cast<IO*>(ws + pl.off_dxdir) + pmine;
 
@@ -542,7 +594,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     for (int i = 0; i < NSTAGE_MAIN; ++i) mbar_init(&full_bar[i], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  for (int e = w.tid; e < 2 * CK * NBC; e += CH) (&red[0][0][0])[e] = 0.f;
+  for (int e = w.tid; e < 2 * CK * NBC; e += NTHR) (&red[0][0][0])[e] = 0.f;
   __syncthreads();
   const uint32_t tx_base = (uint32_t)(CK * CH * ESZ * 2 + CK * CH * 4 + CK * NBC * 4 + TILE_FLOATS * 4 + ncs * 4 +
                                       (WIN ? CK * CH * ESZ + CK * CH * 4 : 0));
@@ -574,31 +626,34 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   if (w.tid == 0)
     for (int i = 0; i < NSTAGE_MAIN && i < nchunk; ++i) issue(i);
 
-  u64 A2[8], mu[8], dAacc[8];
+  u64 A2[NU], mu[NU], dAacc[NU];
   load_A2(A_log, w, A2);
   const int64_t sb = ((int64_t)b * pl.S + s) * pl.tiles + tile;
   load_block_g(reinterpret_cast<const float*>(ws + pl.off_carry) + sb * TILE_FLOATS, w.tid, mu);
   {   // true segment-start state: parked in shared memory, read back once per chunk
-    u64 hst[8];
+    u64 hst[NU];
     load_block_g(reinterpret_cast<const float*>(ws + pl.off_hstart) + sb * TILE_FLOATS, w.tid, hst);
 #pragma unroll
-    for (int q = 0; q < 4; ++q) hst_s[q][w.tid] = make_ulonglong2(hst[2 * q], hst[2 * q + 1]);
+    for (int q = 0; q < 2 * NCH; ++q) hst_s[q][w.tid] = make_ulonglong2(hst[2 * q], hst[2 * q + 1]);
   }
 #pragma unroll
-  for (int u = 0; u < 8; ++u) dAacc[u] = 0ull;
+  for (int u = 0; u < NU; ++u) dAacc[u] = 0ull;
   // least negative exponent scale of each channel over all 16 states (for the window-term skip test)
-  float a2max[2];
+  float a2max[NCH];
 #pragma unroll
-  for (int ch = 0; ch < 2; ++ch) {
+  for (int ch = 0; ch < NCH; ++ch) {
     float mx = -3.0e38f;
 #pragma unroll
     for (int m = 0; m < 4; ++m) { float lo, hi; upk(A2[ch * 4 + m], lo, hi); mx = fmaxf(mx, fmaxf(lo, hi)); }
     a2max[ch] = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
   }
-  double sw[2] = {0.0, 0.0};
+  double sw[NCH];
+#pragma unroll
+  for (int c = 0; c < NCH; ++c) sw[c] = 0.0;
   if (WIN && w.act) {
     const double* swp = reinterpret_cast<const double*>(ws + pl.off_swin) + ((int64_t)b * pl.S + s) * P + w.pa;
-    sw[0] = swp[0]; sw[1] = swp[1];
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) sw[c] = swp[c];
   }
   float dbacc = 0.f;
 
@@ -612,8 +667,9 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     const int rb = i & 1;
     const int nwin = WIN ? (int)max((int64_t)0, min((int64_t)CK, T - tbar - tc)) : 0;   // tokens j < nwin have t + Tbar < T
     // window Delta sum: fp64 value at the chunk's last token + an fp32 running offset inside the chunk
-    const float swc[2] = {(float)sw[0], (float)sw[1]};
-    float swl[2] = {0.f, 0.f};
+    float swc[NCH], swl[NCH];
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) { swc[c] = (float)sw[c]; swl[c] = 0.f; }
     if (nt < CK) {   // only the last chunk of a sequence: neutralise the slots past its end
       if (ok) {
         zero_rows(sm + St::D, CH * 4, nt, w.tid);
@@ -624,14 +680,18 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     }
     if (ok) {
       // state at the chunk start: local checkpoint + decayed true segment-start state
-      u64 h[8];
+      u64 h[NU];
       load_block(reinterpret_cast<const float*>(sm + St::CKP), w.tid, h);
       {
-        float2 csv = *reinterpret_cast<const float2*>(sm + St::CS + 8 * w.k);
-        if (!w.act) csv = make_float2(0.f, 0.f);   // the 1D copy only covers existing channels
-        const u64 c2[2] = {pk(csv.x, csv.x), pk(csv.y, csv.y)};
+        u64 c2[NCH];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
+        for (int c = 0; c < NCH; ++c) {
+          float csv = *reinterpret_cast<const float*>(sm + St::CS + 4 * (NCH * w.k + c));
+          if (!w.act) csv = 0.f;   // the 1D copy only covers existing channels
+          c2[c] = pk(csv, csv);
+        }
+#pragma unroll
+        for (int q = 0; q < 2 * NCH; ++q) {
           const ulonglong2 hq = hst_s[q][w.tid];
           h[2 * q] = fma2(ex2_2(mul2(c2[q / 2], A2[2 * q])), hq.x, h[2 * q]);
           h[2 * q + 1] = fma2(ex2_2(mul2(c2[q / 2], A2[2 * q + 1])), hq.y, h[2 * q + 1]);
@@ -640,7 +700,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
       // forward rebuild in two halves of four tokens (one copy of the code, rolled loop): only the states
       // after tokens 0, 2, 4, 6 are kept; `cur` holds the pair of the half being processed, `hsA` parks the
       // first half's pair while the second half is rebuilt and walked.
-      u64 hsA[2][8], cur[2][8];
+      u64 hsA[2][NU], cur[2][NU];
 #pragma unroll 1
       for (int k = 0; k < 2; ++k) {
         const uint8_t* smk = sm + k * HALF * CH * ESZ;          // x rows of this half
@@ -650,24 +710,28 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         for (int jj = 0; jj < HALF; ++jj) {
           if (jj == HALF - 1 && k == 1) break;                  // the state after the chunk's last token is rebuilt below
           __syncwarp();   // keeps the staged loads of later tokens from being hoisted (register pressure)
-          const float2 dv = lds_pair<float>(smd, jj, w.k);
-          const float2 xv = lds_pair<IO>(smk + St::X, jj, w.k);
+          const ChV dv = lds_ch<float>(smd, jj, w.k);
+          const ChV xv = lds_ch<IO>(smk + St::X, jj, w.k);
           const float* brow = bck + jj * NBC;
           const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
           const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
           const u64 Bp[4] = {b01.x, b01.y, b23.x, b23.y};
-          const u64 d2[2] = {pk(dv.x, dv.x), pk(dv.y, dv.y)};
-          const u64 dx2[2] = {pk(dv.x * xv.x, dv.x * xv.x), pk(dv.y * xv.y, dv.y * xv.y)};
+          u64 d2[NCH], dx2[NCH];
 #pragma unroll
-          for (int u = 0; u < 8; ++u) h[u] = fma2(ex2_2(mul2(d2[u / 4], A2[u])), h[u], mul2(dx2[u / 4], Bp[u % 4]));
+          for (int c = 0; c < NCH; ++c) {
+            const float dxc = dv.v[c] * xv.v[c];
+            d2[c] = pk(dv.v[c], dv.v[c]); dx2[c] = pk(dxc, dxc);
+          }
+#pragma unroll
+          for (int u = 0; u < NU; ++u) h[u] = fma2(ex2_2(mul2(d2[u / 4], A2[u])), h[u], mul2(dx2[u / 4], Bp[u % 4]));
           if ((jj & 1) == 0) {
 #pragma unroll
-            for (int u = 0; u < 8; ++u) cur[jj / 2][u] = h[u];
+            for (int u = 0; u < NU; ++u) cur[jj / 2][u] = h[u];
           }
         }
         if (k == 0) {
 #pragma unroll
-          for (int u = 0; u < 8; ++u) { hsA[0][u] = cur[0][u]; hsA[1][u] = cur[1][u]; }
+          for (int u = 0; u < NU; ++u) { hsA[0][u] = cur[0][u]; hsA[1][u] = cur[1][u]; }
         }
       }
       // backward walk, second half first
@@ -675,7 +739,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
       for (int k = 1; k >= 0; --k) {
         if (k == 0) {
 #pragma unroll
-          for (int u = 0; u < 8; ++u) { cur[0][u] = hsA[0][u]; cur[1][u] = hsA[1][u]; }
+          for (int u = 0; u < NU; ++u) { cur[0][u] = hsA[0][u]; cur[1][u] = hsA[1][u]; }
         }
         const uint8_t* smk = sm + k * HALF * CH * ESZ;          // x / dy rows of this half
         const uint8_t* smd = sm + k * HALF * CH * 4;            // Delta rows
@@ -683,9 +747,9 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
 #pragma unroll
         for (int jj = HALF - 1; jj >= 0; --jj) {
           const int j = k * HALF + jj;
-          const float2 dv = lds_pair<float>(smd + St::D, jj, w.k);
-          const float2 xv = lds_pair<IO>(smk + St::X, jj, w.k);
-          const float2 gv = lds_pair<IO>(smk + St::G, jj, w.k);
+          const ChV dv = lds_ch<float>(smd + St::D, jj, w.k);
+          const ChV xv = lds_ch<IO>(smk + St::X, jj, w.k);
+          const ChV gv = lds_ch<IO>(smk + St::G, jj, w.k);
           const float* brow = bck + St::BC / 4 + jj * NBC;
           const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
           const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
@@ -693,43 +757,53 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
           const ulonglong2 c23 = *reinterpret_cast<const ulonglong2*>(brow + NS + 4);
           const u64 Bp[4] = {b01.x, b01.y, b23.x, b23.y};
           const u64 Cp[4] = {c01.x, c01.y, c23.x, c23.y};
-          const float dd[2] = {dv.x, dv.y}, xs[2] = {xv.x, xv.y}, gs[2] = {gv.x, gv.y};
-          const float dxs[2] = {dv.x * xv.x, dv.y * xv.y};
-          const u64 d2[2] = {pk(dd[0], dd[0]), pk(dd[1], dd[1])};
-          const u64 dx2[2] = {pk(dxs[0], dxs[0]), pk(dxs[1], dxs[1])};
-          const u64 g2[2] = {pk(gs[0], gs[0]), pk(gs[1], gs[1])};
+          float dd[NCH], xs[NCH];
+          u64 d2[NCH], dx2[NCH], g2[NCH];
+#pragma unroll
+          for (int c = 0; c < NCH; ++c) {
+            dd[c] = dv.v[c]; xs[c] = xv.v[c];
+            const float dxc = dv.v[c] * xv.v[c];
+            d2[c] = pk(dd[c], dd[c]); dx2[c] = pk(dxc, dxc); g2[c] = pk(gv.v[c], gv.v[c]);
+          }
           // mu_i += g_i C_i   (mu already carries abar_{i+1} mu_{i+1})
 #pragma unroll
-          for (int u = 0; u < 8; ++u) mu[u] = fma2(g2[u / 4], Cp[u % 4], mu[u]);
+          for (int u = 0; u < NU; ++u) mu[u] = fma2(g2[u / 4], Cp[u % 4], mu[u]);
           if (WIN) {
             // exact exit of token t2 = t + Tbar from the window: subtract W_i gC_{t2},
             // W_i = exp(A * sum_{j=i+1..t2} Delta_j); masked out when t2 >= T
             const float wm = j < nwin ? 1.f : 0.f;
-            float2 d2v = lds_pair<float>(smd + St::D2, jj, w.k);
-            d2v.x *= wm; d2v.y *= wm;
-            const float swf[2] = {swc[0] + swl[0], swc[1] + swl[1]};
+            ChV d2v = lds_ch<float>(smd + St::D2, jj, w.k);
+            float swf[NCH];
             // skip when every factor W = 2^(A2 * sum) of the warp is below 2^-64: the term is then far
             // below one rounding unit of mu
-            const bool live = j < nwin && w.act && (swf[0] * a2max[0] > -64.f || swf[1] * a2max[1] > -64.f);
+            bool live = false;
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+              d2v.v[c] *= wm;
+              swf[c] = swc[c] + swl[c];
+              live = live || (swf[c] * a2max[c] > -64.f);
+            }
+            live = live && j < nwin && w.act;
             if (__any_sync(0xffffffffu, live)) {
-              const float2 g2v = lds_pair<IO>(smk + St::G2, jj, w.k);
+              const ChV g2v = lds_ch<IO>(smk + St::G2, jj, w.k);
               const float* crow = bck + St::BC2 / 4 + jj * NBC + NS;
               const ulonglong2 e01 = *reinterpret_cast<const ulonglong2*>(crow);
               const ulonglong2 e23 = *reinterpret_cast<const ulonglong2*>(crow + 4);
               const u64 C2p[4] = {e01.x, e01.y, e23.x, e23.y};
-              const u64 ng2[2] = {pk(-g2v.x, -g2v.x), pk(-g2v.y, -g2v.y)};
-              const u64 sw2[2] = {pk(swf[0], swf[0]), pk(swf[1], swf[1])};
+              u64 ng2[NCH], sw2[NCH];
 #pragma unroll
-              for (int u = 0; u < 8; ++u)
+              for (int c = 0; c < NCH; ++c) { ng2[c] = pk(-g2v.v[c], -g2v.v[c]); sw2[c] = pk(swf[c], swf[c]); }
+#pragma unroll
+              for (int u = 0; u < NU; ++u)
                 mu[u] = fma2(ex2_2(mul2(sw2[u / 4], A2[u])), mul2(ng2[u / 4], C2p[u % 4]), mu[u]);
             }
-            swl[0] += dd[0] - d2v.x;   // window of token t-1: (t-1, t-1+Tbar]
-            swl[1] += dd[1] - d2v.y;
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) swl[c] += dd[c] - d2v.v[c];   // window of token t-1: (t-1, t-1+Tbar]
           }
           u64 vB[4], vC[4];
-          float ssum[2], dsum[2];
+          float ssum[NCH], dsum[NCH];
 #pragma unroll
-          for (int ch = 0; ch < 2; ++ch) {
+          for (int ch = 0; ch < NCH; ++ch) {
             u64 sacc = 0ull, dacc = 0ull;
 #pragma unroll
             for (int m = 0; m < 4; ++m) {
@@ -751,17 +825,17 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
             dsum[ch] = hsum(dacc);
           }
 #pragma unroll
-          for (int ch = 0; ch < 2; ++ch) {
+          for (int ch = 0; ch < NCH; ++ch) {
             ssum[ch] += __shfl_xor_sync(0xffffffffu, ssum[ch], 1);
             dsum[ch] += __shfl_xor_sync(0xffffffffu, dsum[ch], 1);
           }
           {
-            const float d = w.half ? dd[1] : dd[0], xx = w.half ? xs[1] : xs[0];
-            const float sv = w.half ? ssum[1] : ssum[0], dsv = w.half ? dsum[1] : dsum[0];
+            const float d = dd[chf], xx = xs[chf];
+            const float sv = ssum[chf], dsv = dsum[chf];
             const float ddelta = fmaf(dsv, LN2, xx * sv);
             const float duv = ddelta * sig_from_delta(d);
             dbacc += duv;
-            if (w.act && j < nt) {
+            if (fin && j < nt) {
               const int64_t row = (int64_t)b * T + tc + j;
               st_io<IO>(du + row * du_ld, duv);
               st_io<IO>(dxdir + row * P, d * sv);
@@ -789,14 +863,17 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         }
       }
     }
-    if (WIN) { sw[0] += (double)swl[0]; sw[1] += (double)swl[1]; }
+    if (WIN) {
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) sw[c] += (double)swl[c];
+    }
     const int bad = __syncthreads_or(ok ? 0 : 1);
     if (bad) {
       if (w.tid == 0) atomicExch(status, AS_ERR_TIMEOUT);
       return;
     }
     if (w.tid == 0 && i + NSTAGE_MAIN < nchunk) issue(i + NSTAGE_MAIN);
-    for (int e = w.tid; e < CK * NBC; e += CH) {
+    for (int e = w.tid; e < CK * NBC; e += NTHR) {
       const int j = e / NBC, q = e % NBC;
       const float sum = red[rb][j][q];
       red[rb][j][q] = 0.f;   // ready for the chunk after next
@@ -805,7 +882,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   }
   if (w.act) {
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
+    for (int u = 0; u < NU; ++u) {
       float alo, ahi, vlo, vhi;
       upk(A2[u], alo, ahi);
       upk(dAacc[u], vlo, vhi);
@@ -813,8 +890,8 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
       atomicAdd(dst, vlo * (alo * LN2));
       atomicAdd(dst + 1, vhi * (ahi * LN2));
     }
-    atomicAdd(db_delta + pmine, dbacc);
   }
+  if (fin) atomicAdd(db_delta + pmine, dbacc);
 }
 
 template <typename IO>
@@ -875,7 +952,7 @@ int launch_ascend_t(const Plan& pl, const ScanPtrs& sp, void* y, cudaStream_t st
   auto kern = ascend_kernel<IO, MODE>;
   static bool once = false;
   if (!once) { if (set_smem(kern, bytes)) return 1; once = true; }
-  kern<<<dim3(pl.tiles, pl.S, pl.B), CH, bytes, st>>>(m.x, m.d, m.g, pl, sp.A_log, sp.ws, (IO*)y);
+  kern<<<dim3(pl.tiles, pl.S, pl.B), NTHR, bytes, st>>>(m.x, m.d, m.g, pl, sp.A_log, sp.ws, (IO*)y);
   count_launch();
   return (int)cudaGetLastError();
 }
@@ -889,7 +966,7 @@ int launch_main_t(const Plan& pl, const ScanPtrs& sp, float* dA_log, float* db_d
   auto kern = adjoint_main_kernel<IO, FULL>;
   static bool once = false;
   if (!once) { if (set_smem(kern, bytes)) return 1; once = true; }
-  kern<<<dim3(pl.tiles, pl.S, pl.B), CH, bytes, st>>>(m.x, m.d, m.g, pl, sp.A_log, sp.ws, dA_log, db_delta);
+  kern<<<dim3(pl.tiles, pl.S, pl.B), NTHR, bytes, st>>>(m.x, m.d, m.g, pl, sp.A_log, sp.ws, dA_log, db_delta);
   count_launch();
   return (int)cudaGetLastError();
 }
@@ -907,10 +984,10 @@ int launch_prepass(const Plan& pl, const ScanPtrs& sp, bool with_mu, cudaStream_
 }
 
 int launch_fixup(const Plan& pl, const ScanPtrs& sp, bool with_mu, cudaStream_t st) {
-  fixup_h_kernel<<<dim3(pl.tiles, pl.B), CH, 0, st>>>(pl, sp.A_log, sp.ws);
+  fixup_h_kernel<<<dim3(pl.tiles, pl.B), NTHR, 0, st>>>(pl, sp.A_log, sp.ws);
   count_launch();
   if (with_mu) {
-    fixup_mu_kernel<<<dim3(pl.tiles, pl.full ? 1 : pl.S, pl.B), CH, 0, st>>>(pl, sp.A_log, sp.ws);
+    fixup_mu_kernel<<<dim3(pl.tiles, pl.full ? 1 : pl.S, pl.B), NTHR, 0, st>>>(pl, sp.A_log, sp.ws);
     count_launch();
   }
   return (int)cudaGetLastError();
