@@ -667,9 +667,10 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     const int rb = i & 1;
     const int nwin = WIN ? (int)max((int64_t)0, min((int64_t)CK, T - tbar - tc)) : 0;   // tokens j < nwin have t + Tbar < T
     // window Delta sum: fp64 value at the chunk's last token + an fp32 running offset inside the chunk
-    float swc[NCH], swl[NCH];
+    float swc[NCH], swl[NCH], dsumc[NCH], sd2[NCH];
 #pragma unroll
-    for (int c = 0; c < NCH; ++c) { swc[c] = (float)sw[c]; swl[c] = 0.f; }
+    for (int c = 0; c < NCH; ++c) { swc[c] = (float)sw[c]; swl[c] = 0.f; dsumc[c] = 0.f; sd2[c] = 0.f; }
+    bool chunk_live = false;   // warp-uniform: does any exit factor W of this chunk reach 2^-64 ?
     if (nt < CK) {   // only the last chunk of a sequence: neutralise the slots past its end
       if (ok) {
         zero_rows(sm + St::D, CH * 4, nt, w.tid);
@@ -696,6 +697,22 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
           h[2 * q] = fma2(ex2_2(mul2(c2[q / 2], A2[2 * q])), hq.x, h[2 * q]);
           h[2 * q + 1] = fma2(ex2_2(mul2(c2[q / 2], A2[2 * q + 1])), hq.y, h[2 * q + 1]);
         }
+      }
+      if (WIN) {
+        // Delta of the tokens leaving the window during this chunk.  Inside the chunk the window sum never drops
+        // below (sum at the chunk's last token) - (their total), so if even that bound gives W < 2^-64 for every
+        // state of every lane, the exit terms of the whole chunk are skipped: they are far below one rounding unit
+        // of mu.  The decision is taken once per chunk and per warp.
+#pragma unroll
+        for (int j = 0; j < CK; ++j) {
+          const ChV d2v = lds_ch<float>(sm + St::D2, j, w.k);
+#pragma unroll
+          for (int c = 0; c < NCH; ++c) sd2[c] += j < nwin ? d2v.v[c] : 0.f;
+        }
+        bool live = false;
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) live = live || ((swc[c] - sd2[c]) * a2max[c] > -64.f);
+        chunk_live = __any_sync(0xffffffffu, live && w.act && nwin > 0);
       }
       // forward rebuild in two halves of four tokens (one copy of the code, rolled loop): only the states
       // after tokens 0, 2, 4, 6 are kept; `cur` holds the pair of the half being processed, `hsA` parks the
@@ -734,6 +751,9 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
           for (int u = 0; u < NU; ++u) { hsA[0][u] = cur[0][u]; hsA[1][u] = cur[1][u]; }
         }
       }
+      // output rows of this chunk, walked from its last token down
+      IO* du_p = du + ((int64_t)b * T + tc + (CK - 1)) * du_ld;
+      IO* dx_p = dxdir + ((int64_t)b * T + tc + (CK - 1)) * P;
       // backward walk, second half first
 #pragma unroll 1
       for (int k = 1; k >= 0; --k) {
@@ -768,37 +788,31 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
           // mu_i += g_i C_i   (mu already carries abar_{i+1} mu_{i+1})
 #pragma unroll
           for (int u = 0; u < NU; ++u) mu[u] = fma2(g2[u / 4], Cp[u % 4], mu[u]);
-          if (WIN) {
+#pragma unroll
+          for (int c = 0; c < NCH; ++c) dsumc[c] += dd[c];
+          if (WIN && chunk_live) {
             // exact exit of token t2 = t + Tbar from the window: subtract W_i gC_{t2},
             // W_i = exp(A * sum_{j=i+1..t2} Delta_j); masked out when t2 >= T
             const float wm = j < nwin ? 1.f : 0.f;
-            ChV d2v = lds_ch<float>(smd + St::D2, jj, w.k);
-            float swf[NCH];
-            // skip when every factor W = 2^(A2 * sum) of the warp is below 2^-64: the term is then far
-            // below one rounding unit of mu
-            bool live = false;
+            const ChV d2v = lds_ch<float>(smd + St::D2, jj, w.k);
+            const ChV g2v = lds_ch<IO>(smk + St::G2, jj, w.k);
+            const float* crow = bck + St::BC2 / 4 + jj * NBC + NS;
+            const ulonglong2 e01 = *reinterpret_cast<const ulonglong2*>(crow);
+            const ulonglong2 e23 = *reinterpret_cast<const ulonglong2*>(crow + 4);
+            // rows of tokens past the sequence end are not staged: their C values must not be touched
+            const u64 C2p[4] = {wm != 0.f ? e01.x : 0ull, wm != 0.f ? e01.y : 0ull, wm != 0.f ? e23.x : 0ull,
+                                wm != 0.f ? e23.y : 0ull};
+            u64 ng2[NCH], sw2[NCH];
 #pragma unroll
             for (int c = 0; c < NCH; ++c) {
-              d2v.v[c] *= wm;
-              swf[c] = swc[c] + swl[c];
-              live = live || (swf[c] * a2max[c] > -64.f);
-            }
-            live = live && j < nwin && w.act;
-            if (__any_sync(0xffffffffu, live)) {
-              const ChV g2v = lds_ch<IO>(smk + St::G2, jj, w.k);
-              const float* crow = bck + St::BC2 / 4 + jj * NBC + NS;
-              const ulonglong2 e01 = *reinterpret_cast<const ulonglong2*>(crow);
-              const ulonglong2 e23 = *reinterpret_cast<const ulonglong2*>(crow + 4);
-              const u64 C2p[4] = {e01.x, e01.y, e23.x, e23.y};
-              u64 ng2[NCH], sw2[NCH];
-#pragma unroll
-              for (int c = 0; c < NCH; ++c) { ng2[c] = pk(-g2v.v[c], -g2v.v[c]); sw2[c] = pk(swf[c], swf[c]); }
-#pragma unroll
-              for (int u = 0; u < NU; ++u)
-                mu[u] = fma2(ex2_2(mul2(sw2[u / 4], A2[u])), mul2(ng2[u / 4], C2p[u % 4]), mu[u]);
+              const float swf = swc[c] + swl[c];
+              ng2[c] = pk(-g2v.v[c] * wm, -g2v.v[c] * wm);
+              sw2[c] = pk(swf, swf);
+              swl[c] += dd[c] - d2v.v[c] * wm;   // window of token t-1: (t-1, t-1+Tbar]
             }
 #pragma unroll
-            for (int c = 0; c < NCH; ++c) swl[c] += dd[c] - d2v.v[c];   // window of token t-1: (t-1, t-1+Tbar]
+            for (int u = 0; u < NU; ++u)
+              mu[u] = fma2(ex2_2(mul2(sw2[u / 4], A2[u])), mul2(ng2[u / 4], C2p[u % 4]), mu[u]);
           }
           u64 vB[4], vC[4];
           float ssum[NCH], dsum[NCH];
@@ -836,10 +850,11 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
             const float duv = ddelta * sig_from_delta(d);
             dbacc += duv;
             if (fin && j < nt) {
-              const int64_t row = (int64_t)b * T + tc + j;
-              st_io<IO>(du + row * du_ld, duv);
-              st_io<IO>(dxdir + row * P, d * sv);
+              st_io<IO>(du_p, duv);
+              st_io<IO>(dx_p, d * sv);
             }
+            du_p -= du_ld;
+            dx_p -= P;
           }
           // sum over the warp's 16 channel pairs: every lane parks its 16 partials (dB[8*half+0..7], dC[8*half+0..7])
           // in shared memory, then lane l adds up value (l >> 1) over the 16 lanes of its parity.  Quarter-blocks
@@ -849,8 +864,8 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
             __syncwarp();   // the previous token's loads from wr are done
 #pragma unroll
             for (int m = 0; m < 4; ++m) {
-              const u64* src = (m < 2) ? &vB[2 * m] : &vC[2 * (m - 2)];
-              *reinterpret_cast<ulonglong2*>(wr + m * WRED_Q + lane * 4) = make_ulonglong2(src[0], src[1]);
+              *reinterpret_cast<u64*>(wr + (m >> 1) * WRED_Q + lane * 4 + 2 * (m & 1)) = vB[m];
+              *reinterpret_cast<u64*>(wr + (2 + (m >> 1)) * WRED_Q + lane * 4 + 2 * (m & 1)) = vC[m];
             }
             __syncwarp();
             const int vi = lane >> 1;
@@ -865,8 +880,9 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     }
     if (WIN) {
 #pragma unroll
-      for (int c = 0; c < NCH; ++c) sw[c] += (double)swl[c];
+      for (int c = 0; c < NCH; ++c) sw[c] += (double)(dsumc[c] - sd2[c]);   // window sum at the previous chunk's last token
     }
+    (void)swl;
     const int bad = __syncthreads_or(ok ? 0 : 1);
     if (bad) {
       if (w.tid == 0) atomicExch(status, AS_ERR_TIMEOUT);
