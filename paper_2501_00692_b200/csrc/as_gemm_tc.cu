@@ -15,7 +15,7 @@
 namespace as {
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 64, STAGES = 6, UK = 16, NTHREADS = 192;
+constexpr int BM = 128, BN = 128, BK = 64, STAGES = 6, UK = 16, EPI_WARPS = 8, NTHREADS = 64 + 32 * EPI_WARPS;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int SMEM_DYN = STAGES * STAGE_BYTES + 1024;  // + slack for 1024-byte alignment
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
@@ -122,7 +122,8 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 // Persistent, warp-specialised kernel: one CTA per SM walks tiles t = blockIdx.x, + gridDim.x, ...
 //   warp 0 (one lane): TMA producer over a STAGES-deep shared-memory ring that runs on across tiles
 //   warp 1 (one lane): tcgen05.mma issuer; the accumulator alternates between two 128-column TMEM buffers
-//   warps 2..5       : epilogue; drain buffer a while the issuer already fills buffer a^1 for the next tile
+//   warps 2..9       : epilogue (two warps per TMEM lane quarter, each taking half of the columns); they drain
+//                      buffer a while the issuer already fills buffer a^1 for the next tile
 // Tile order: n fastest, then m, then the K split, so concurrently running CTAs share A rows through L2.
 template <int AMAJ, int BMAJ, int EPI>
 __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
@@ -144,7 +145,7 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full_bar[b], 1); mbar_init(&tmem_empty_bar[b], 4); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full_bar[b], 1); mbar_init(&tmem_empty_bar[b], EPI_WARPS); }
     abort_s = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -234,7 +235,9 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
     }
   } else {
     // ---------------- epilogue warps ----------------
-    const int quarter = warp & 3;   // the TMEM lane quarter this warp may read
+    const int quarter = warp & 3;              // the TMEM lane quarter this warp may read
+    const int chalf = (warp - 2) / 4;          // which half of the tile's columns it drains
+    constexpr int CPW = BN / 32 / (EPI_WARPS / 4);   // 32-column chunks per warp
     int ti = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++ti) {
@@ -246,7 +249,7 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const int64_t m = m0 + quarter * 32 + lane;   // this thread's output row
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
+        for (int c = chalf * CPW; c < (chalf + 1) * CPW; ++c) {
           uint32_t r[32];
           tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(ab * BN + c * 32), r);
           const int nb = n0 + c * 32;
