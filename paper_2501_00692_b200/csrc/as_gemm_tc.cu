@@ -15,9 +15,16 @@
 namespace as {
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 64, STAGES = 6, UK = 16, EPI_WARPS = 8, NTHREADS = 64 + 32 * EPI_WARPS;
-constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int SMEM_DYN = STAGES * STAGE_BYTES + 1024;  // + slack for 1024-byte alignment
+constexpr int BM = 128, BK = 64, UK = 16, EPI_WARPS = 8, NTHREADS = 64 + 32 * EPI_WARPS;
+constexpr int A_BYTES = BM * BK * 2;
+// tile width BN is a template parameter: 256 keeps the shared-memory operand traffic per MMA cycle under the
+// 128 B/clk an SM can read (a 128x128 tile needs 128 B/clk for the MMA alone), 128 wastes less on narrow outputs
+template <int BN> struct Cfg {
+  static constexpr int B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int STAGES = BN >= 208 ? 4 : 6;
+  static constexpr int TMEM_COLS = 2 * BN <= 256 ? 256 : 512;   // two accumulators, power-of-two allocation
+  static constexpr int SMEM_DYN = STAGES * STAGE_BYTES + 1024;   // + slack for 1024-byte alignment
+};
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
 enum { MAJ_K = 0, MAJ_MN = 1 };
@@ -104,6 +111,15 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
 // softplus(u) = max(u,0) + log(1 + z), z = exp(-|u|) in (0,1]: two MUFU ops (ex2, lg2) and a short series
 // for small z, where forming 1 + z would lose z's low bits (relative error of the result < 3e-7)
 __device__ __forceinline__ float softplus_f(float u) {
@@ -125,9 +141,10 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 //   warps 2..9       : epilogue (two warps per TMEM lane quarter, each taking half of the columns); they drain
 //                      buffer a while the issuer already fills buffer a^1 for the next tile
 // Tile order: n fastest, then m, then the K split, so concurrently running CTAs share A rows through L2.
-template <int AMAJ, int BMAJ, int EPI>
+template <int AMAJ, int BMAJ, int EPI, int BN>
 __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
                                                            const __grid_constant__ CUtensorMap tmB, TcArgs a) {
+  constexpr int STAGES = Cfg<BN>::STAGES, B_BYTES = Cfg<BN>::B_BYTES, STAGE_BYTES = Cfg<BN>::STAGE_BYTES;
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[STAGES];
   __shared__ __align__(8) uint64_t empty_bar[STAGES];
@@ -150,7 +167,7 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {   // TMEM allocation: two BN-column fp32 accumulators
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(2 * BN)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(Cfg<BN>::TMEM_COLS)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -192,8 +209,8 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
           if (BMAJ == MAJ_K) {
             tma_load_2d(sb, &tmB, k, n0, &full_bar[s]);
           } else {
-            tma_load_2d(sb, &tmB, n0, k, &full_bar[s]);
-            tma_load_2d(sb + B_BYTES / 2, &tmB, n0 + 64, k, &full_bar[s]);
+#pragma unroll
+            for (int q = 0; q < BN / 64; ++q) tma_load_2d(sb + q * (64 * BK * 2), &tmB, n0 + 64 * q, k, &full_bar[s]);
           }
         }
       }
@@ -202,8 +219,8 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
   } else if (warp == 1) {
     if (lane == 0) {
       // ---------------- MMA issuer ----------------
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)AMAJ << 15) | ((uint32_t)BMAJ << 16) |
-                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      const uint32_t idesc0 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)AMAJ << 15) | ((uint32_t)BMAJ << 16) |
+                              ((uint32_t)(BM >> 4) << 24);
       int it = 0, ti = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++ti) {
@@ -213,6 +230,10 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
         if (around > 0 && !mbar_wait(&tmem_empty_bar[ab], (around - 1) & 1, abortp)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t acc = tmem_base + (uint32_t)(ab * BN);
+        // a K-major B tile that sticks out past N only needs the MMA to cover its valid columns (multiple of 16)
+        int neff = BN;
+        if (BMAJ == MAJ_K && n0 + BN > a.N) neff = ((a.N - n0 + 15) / 16) * 16;
+        const uint32_t idesc = idesc0 | ((uint32_t)(neff >> 3) << 17);
         for (int i = 0; i < nkb; ++i, ++it) {
           const int s = it % STAGES, round = it / STAGES;
           if (!mbar_wait(&full_bar[s], round & 1, abortp)) { ok = false; break; }
@@ -224,7 +245,7 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
             const uint64_t ad = (AMAJ == MAJ_K) ? make_desc(sa + k * UK * 2, 16, 1024)
                                                 : make_desc(sa + k * UK * 128, A_BYTES / 2, 1024);
             const uint64_t bd = (BMAJ == MAJ_K) ? make_desc(sb + k * UK * 2, 16, 1024)
-                                                : make_desc(sb + k * UK * 128, B_BYTES / 2, 1024);
+                                                : make_desc(sb + k * UK * 128, 64 * BK * 2, 1024);
             umma_bf16(acc, ad, bd, idesc, (i > 0 || k > 0) ? 1u : 0u);
           }
           umma_commit(&empty_bar[s]);   // frees the stage once these MMAs have read it
@@ -237,7 +258,8 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
     // ---------------- epilogue warps ----------------
     const int quarter = warp & 3;              // the TMEM lane quarter this warp may read
     const int chalf = (warp - 2) / 4;          // which half of the tile's columns it drains
-    constexpr int CPW = BN / 32 / (EPI_WARPS / 4);   // 32-column chunks per warp
+    constexpr int NCHUNK = BN / 16;                            // 16-column chunks of a tile
+    constexpr int CSPLIT = (NCHUNK + 1) / 2;                   // first warp of a quarter takes [0, CSPLIT)
     int ti = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++ti) {
@@ -249,17 +271,17 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const int64_t m = m0 + quarter * 32 + lane;   // this thread's output row
 #pragma unroll 1
-        for (int c = chalf * CPW; c < (chalf + 1) * CPW; ++c) {
-          uint32_t r[32];
-          tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(ab * BN + c * 32), r);
-          const int nb = n0 + c * 32;
+        for (int c = chalf ? CSPLIT : 0; c < (chalf ? NCHUNK : CSPLIT); ++c) {
+          uint32_t r[16];
+          tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(ab * BN + c * 16), r);
+          const int nb = n0 + c * 16;
           if (m >= a.M || nb >= a.N) continue;
           if (EPI == TC_PROJ) {
             if (nb < a.P) {
               float4* dst = reinterpret_cast<float4*>(a.delta + m * a.P + nb);
               const float4* b4 = reinterpret_cast<const float4*>(a.bias + nb);
 #pragma unroll
-              for (int q = 0; q < 8; ++q) {
+              for (int q = 0; q < 4; ++q) {
                 const float4 bv = __ldg(b4 + q);
                 dst[q] = make_float4(softplus_f(__uint_as_float(r[4 * q]) + bv.x), softplus_f(__uint_as_float(r[4 * q + 1]) + bv.y),
                                      softplus_f(__uint_as_float(r[4 * q + 2]) + bv.z), softplus_f(__uint_as_float(r[4 * q + 3]) + bv.w));
@@ -267,7 +289,7 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
             } else {
               float4* dst = reinterpret_cast<float4*>(a.bc + m * NBC + (nb - a.P));
 #pragma unroll
-              for (int q = 0; q < 8; ++q)
+              for (int q = 0; q < 4; ++q)
                 dst[q] = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]), __uint_as_float(r[4 * q + 2]),
                                      __uint_as_float(r[4 * q + 3]));
             }
@@ -277,12 +299,12 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
             else if (m < a.P + NS) dst = a.dW_B + (m - a.P) * a.P + nb;
             else dst = a.dW_C + (m - a.P - NS) * a.P + nb;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) atomicAdd(dst + j, __uint_as_float(r[j]));
+            for (int j = 0; j < 16; ++j) atomicAdd(dst + j, __uint_as_float(r[j]));
           } else {
             const uint4* src = reinterpret_cast<const uint4*>(a.dxdir + m * a.P + nb);
             uint4* dst = reinterpret_cast<uint4*>(a.dx + m * a.P + nb);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
+            for (int q = 0; q < 2; ++q) {
               const uint4 sv = __ldg(src + q);
               const __nv_bfloat162* s2 = reinterpret_cast<const __nv_bfloat162*>(&sv);
               uint4 ov;
@@ -307,7 +329,7 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (warp == 1) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * BN) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(Cfg<BN>::TMEM_COLS) : "memory");
   }
 }
 
@@ -359,22 +381,25 @@ int make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, ui
   return r == CUDA_SUCCESS ? 0 : 1;
 }
 
-template <int AMAJ, int BMAJ, int EPI>
+template <int AMAJ, int BMAJ, int EPI, int BN>
 int launch_tc(const CUtensorMap& tmA, const CUtensorMap& tmB, const TcArgs& a, cudaStream_t st) {
   static bool attr_set = false;
-  auto kern = gemm_tc_kernel<AMAJ, BMAJ, EPI>;
+  auto kern = gemm_tc_kernel<AMAJ, BMAJ, EPI, BN>;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN) != cudaSuccess) return 1;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::SMEM_DYN) != cudaSuccess) return 1;
     attr_set = true;
   }
   const int64_t ntiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN) * a.splitk;
   const unsigned grid = (unsigned)(ntiles < 148 ? ntiles : 148);   // one persistent CTA per SM
-  kern<<<grid, NTHREADS, SMEM_DYN, st>>>(tmA, tmB, a);
+  kern<<<grid, NTHREADS, Cfg<BN>::SMEM_DYN, st>>>(tmA, tmB, a);
   count_launch();
   return (int)cudaGetLastError();
 }
 
 }  // namespace
+
+constexpr int TBN = 256;   // tile width of the weight-gradient and input-gradient contractions
+constexpr int PBN = 208;   // projections: N = P + 32; for P = 768 four 208-wide tiles waste 4 % where 256 wastes 22 %
 
 int tc_pack_wcat(const Plan& pl, const as_params_t* pr, char* ws, cudaStream_t st) {
   const int64_t n = (int64_t)(pl.P + NBC) * pl.P;
@@ -390,12 +415,12 @@ int tc_projections(const Plan& pl, const as_params_t* pr, const void* x, char* w
   const int P = pl.P, NW = P + NBC;
   CUtensorMap tmA, tmB;
   if (make_map(&tmA, x, M, P, P, BM)) return 1;
-  if (make_map(&tmB, ws + pl.off_wcat, NW, P, P, BN)) return 1;
+  if (make_map(&tmB, ws + pl.off_wcat, NW, P, P, PBN)) return 1;
   TcArgs a{};
   a.M = M; a.N = NW; a.kblocks = (P + BK - 1) / BK; a.splitk = 1; a.P = P;
   a.delta = (float*)(ws + pl.off_delta); a.bc = (float*)(ws + pl.off_bc); a.bias = pr->b_delta;
   a.status = (int*)(ws + pl.off_status);
-  return launch_tc<MAJ_K, MAJ_K, TC_PROJ>(tmA, tmB, a, st);
+  return launch_tc<MAJ_K, MAJ_K, TC_PROJ, PBN>(tmA, tmB, a, st);
 }
 
 int tc_weight_grads(const Plan& pl, const void* x, const as_grads_t* out, char* ws, cudaStream_t st) {
@@ -410,7 +435,7 @@ int tc_weight_grads(const Plan& pl, const void* x, const as_grads_t* out, char* 
   if (make_map(&tmB, x, M, P, P, 64)) return 1;                  // X as [K=tokens, N=P]
   TcArgs a{};
   a.M = NW; a.N = P; a.kblocks = (int)((M + BK - 1) / BK); a.P = P;
-  const int tiles = ((NW + BM - 1) / BM) * ((P + BN - 1) / BN);
+  const int tiles = ((NW + BM - 1) / BM) * ((P + TBN - 1) / TBN);
   int sk = (148 * 2) / tiles;   // about two tiles per persistent CTA
   if (sk > a.kblocks) sk = a.kblocks;
   if (sk < 1) sk = 1;
@@ -418,7 +443,7 @@ int tc_weight_grads(const Plan& pl, const void* x, const as_grads_t* out, char* 
   a.splitk = (a.kblocks + kper - 1) / kper;   // no empty split: every tile has at least one K block
   a.dW_delta = out->dW_delta; a.dW_B = out->dW_B; a.dW_C = out->dW_C;
   a.status = (int*)(ws + pl.off_status);
-  return launch_tc<MAJ_MN, MAJ_MN, TC_DW>(tmA, tmB, a, st);
+  return launch_tc<MAJ_MN, MAJ_MN, TC_DW, TBN>(tmA, tmB, a, st);
 }
 
 int tc_input_grad(const Plan& pl, void* dx, char* ws, cudaStream_t st) {
@@ -431,7 +456,7 @@ int tc_input_grad(const Plan& pl, void* dx, char* ws, cudaStream_t st) {
   a.M = M; a.N = P; a.kblocks = (NW + BK - 1) / BK; a.splitk = 1; a.P = P;
   a.dxdir = (const __nv_bfloat16*)(ws + pl.off_dxdir); a.dx = (__nv_bfloat16*)dx;
   a.status = (int*)(ws + pl.off_status);
-  return launch_tc<MAJ_K, MAJ_MN, TC_DX>(tmA, tmB, a, st);
+  return launch_tc<MAJ_K, MAJ_MN, TC_DX, TBN>(tmA, tmB, a, st);
 }
 
 }  // namespace as
