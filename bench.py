@@ -76,7 +76,7 @@ class ClockSampler:
             except (ValueError, IndexError):
                 continue
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "sm_mhz_min": min(sm) if sm else None}
 
 
 def max_over_ranks(values, device, world):
@@ -141,7 +141,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C3")
@@ -192,14 +192,13 @@ def main():
     def step():
         B.as_adjoint_grad(sh, theta, x, dy, w.tbar, grads, ws)
 
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()        # samples SM clocks / throttle reasons from here to the end of the timed regions
     for _ in range(args.warmup):
         step()
     torch.cuda.synchronize()
     assert B.as_check_status(ws) == 0
-
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
     # ---- device-resident timing --------------------------------------------------------------
     B.as_launch_count(reset=True)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -219,13 +218,13 @@ def main():
         for k, v in B.as_get_timing().items():
             phase[k] += v / args.steps
     B.as_set_timing(False)
-    clocks = sampler.stop() if rank == 0 else None
     # ---- end to end: pinned host inputs -> device, gradients -> host, inside the timed region -----
     if args.no_e2e:
         ms_e2e, h2d, d2h = float("nan"), 0, 0
     else:
         ms_e2e, h2d, d2h = run_e2e(args, torch, x, dy, grads, step, barrier, e0, e1)
 
+    clocks = sampler.stop() if rank == 0 else None
     ms, ms_e2e = max_over_ranks([ms, ms_e2e if ms_e2e == ms_e2e else -1.0], dev, world)
     if ms_e2e < 0:
         ms_e2e = float("nan")
