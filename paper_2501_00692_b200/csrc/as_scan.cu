@@ -870,9 +870,14 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
             __syncwarp();
             const int vi = lane >> 1;
             const float* rd = wr + (vi >> 2) * WRED_Q + (lane & 1) * 4 + (vi & 3);
-            float tot = 0.f;
+            float part[16];
 #pragma unroll
-            for (int i2 = 0; i2 < 16; ++i2) tot += rd[i2 * 8];
+            for (int i2 = 0; i2 < 16; ++i2) part[i2] = rd[i2 * 8];
+#pragma unroll
+            for (int wdt = 8; wdt >= 1; wdt >>= 1)   // pairwise tree: 4 dependent adds instead of 16
+#pragma unroll
+              for (int i2 = 0; i2 < wdt; ++i2) part[i2] += part[i2 + wdt];
+            const float tot = part[0];
             atomicAdd(&red[rb][j][(vi & 8) * 2 + 8 * w.half + (vi & 7)], tot);
           }
         }
