@@ -276,7 +276,9 @@ def report(args, B, w, world, rank, tokens, ms, ms_e2e, h2d, d2h, launches, phas
     if rank == 0:
         peak, peak_src = measured_peaks()
         e = 2 if w.io == "bf16" else 4
-        bytes_per_token = w.d_model * (2 * e + 4 + 2 * e) + 2 * (2 * w.d_state * 4)   # see the design doc, adjoint main kernel
+        # algorithmic bytes of the main adjoint kernel per token: read x, dy (2 P e) and Delta (4 P); write du, dx_dir (2 P e);
+        # read [B|C] and write [dB|dC] (2 x 2N fp32)
+        bytes_per_token = w.d_model * (2 * e + 4 + 2 * e) + 2 * (2 * w.d_state * 4)
         k_ms = phase["adjoint_main"]
         achieved = bytes_per_token * tokens / (k_ms * 1e-3) / 1e9 if k_ms > 0 else None
         # MUFU issue bound of the same kernel: >= 2 ex2 per (token, channel, state) in the chunk walk + 1/8 for the
