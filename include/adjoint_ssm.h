@@ -143,7 +143,16 @@ int as_residual_add(const as_shape_t *shape, const void *y_in, const void *ytild
 int as_rmsnorm_bwd_add(const as_shape_t *shape, const void *y, const void *dyhat, void *G_inout,
                        float eps, void *stream);
 
-/* ---- diagnostics (host-side bookkeeping only; no effect on results) ------------------------------ */
+/* ---- diagnostics ------------------------------------------------------------------------------------ */
+
+/* Self test of the failure-reporting path.  Every device-side wait of this library (mbarrier waits on staged
+ * tiles) is bounded: after a fixed number of polls the kernel stops, writes AS_ERR_TIMEOUT into the status word at
+ * the head of `ws` and returns, leaving the context usable.  This call enqueues a one-warp kernel that waits, with
+ * `poll_limit` polls (1 .. 2^20), for an mbarrier phase that nothing completes; as_check_status(ws, stream) must
+ * then return AS_ERR_TIMEOUT.  `ws` needs 256 bytes.  Nothing faults, traps or spins without bound. */
+int as_wait_selftest(void *ws, size_t ws_bytes, uint32_t poll_limit, void *stream);
+
+/* host-side bookkeeping only; no effect on results */
 
 /* Number of kernels this library has launched in this process since the last reset; reset != 0 zeroes it. */
 int64_t as_launch_count(int reset);

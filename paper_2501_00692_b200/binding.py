@@ -22,7 +22,7 @@ AS_ERR_WORKSPACE, AS_ERR_ALIGN, AS_ERR_CUDA, AS_ERR_TIMEOUT, AS_ERR_LIMIT = -5, 
 
 EXPORTS = ("as_version", "as_strerror", "as_workspace_bytes", "as_check_status", "as_ssm_forward",
            "as_adjoint_grad", "as_full_bptt_grad", "as_rmsnorm_fwd", "as_residual_add", "as_rmsnorm_bwd_add",
-           "as_launch_count", "as_set_timing", "as_get_timing", "as_ssm_forward_static")
+           "as_launch_count", "as_set_timing", "as_get_timing", "as_ssm_forward_static", "as_wait_selftest")
 AS_STATIC_SCRATCH_BYTES = 32 << 20
 AS_NUM_PHASES = 6
 PHASES = ("projections", "prepass", "fixup", "adjoint_main", "weight_grads", "input_grad")
@@ -77,6 +77,7 @@ def lib() -> C.CDLL:
                                          C.c_void_p]
         L.as_ssm_forward_static.argtypes = [C.POINTER(as_shape_t), C.POINTER(as_params_t), C.c_void_p, C.c_void_p,
                                             C.c_void_p]
+        L.as_wait_selftest.argtypes = [C.c_void_p, C.c_size_t, C.c_uint32, C.c_void_p]
         L.as_launch_count.argtypes = [C.c_int]
         L.as_set_timing.argtypes = [C.c_int]
         L.as_get_timing.argtypes = [C.POINTER(C.c_float), C.c_int]
@@ -212,3 +213,8 @@ def as_ssm_forward_static(shape, theta, x, y, stream=None):
     p = make_params(theta)
     _check(lib().as_ssm_forward_static(C.byref(shape), C.byref(p), _ptr(x), _ptr(y), _stream(stream)),
            "as_ssm_forward_static")
+
+
+def as_wait_selftest(ws, poll_limit=4096, stream=None):
+    """Enqueue the bounded-wait self test; afterwards as_check_status(ws) must return AS_ERR_TIMEOUT."""
+    _check(lib().as_wait_selftest(_ptr(ws), ws.numel(), int(poll_limit), _stream(stream)), "as_wait_selftest")

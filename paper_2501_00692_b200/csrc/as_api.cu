@@ -291,6 +291,17 @@ int as_rmsnorm_bwd_add(const as_shape_t* shape, const void* y, const void* dyhat
   return AS_OK;
 }
 
+int as_wait_selftest(void* ws, size_t ws_bytes, uint32_t poll_limit, void* stream) {
+  if (!ws) return AS_ERR_NULL;
+  if (ws_bytes < 256) return AS_ERR_WORKSPACE;
+  if (!aligned16(ws)) return AS_ERR_ALIGN;
+  if (poll_limit == 0 || poll_limit > (1u << 20)) return AS_ERR_LIMIT;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  AS_TRY((int)cudaMemsetAsync(ws, 0, 256, st));
+  AS_TRY(launch_wait_selftest(reinterpret_cast<int*>(ws), poll_limit, st));
+  return AS_OK;
+}
+
 int64_t as_launch_count(int reset) {
   const int64_t v = as::g_launches.load();
   if (reset) as::g_launches.store(0);

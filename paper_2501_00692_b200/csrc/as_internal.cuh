@@ -96,6 +96,7 @@ int launch_prepass(const Plan& pl, const ScanPtrs& sp, bool with_mu, cudaStream_
 int launch_fixup(const Plan& pl, const ScanPtrs& sp, bool with_mu, cudaStream_t st);
 int launch_forward_y(const Plan& pl, const ScanPtrs& sp, void* y, cudaStream_t st);
 int launch_adjoint_main(const Plan& pl, const ScanPtrs& sp, float* dA_log, float* db_delta, cudaStream_t st);
+int launch_wait_selftest(int* status, unsigned limit, cudaStream_t st);
 int launch_finish_dx(const Plan& pl, const float* dxacc, const void* dxdir, void* dx, cudaStream_t st);
 
 // bf16 tensor-core path (as_gemm_tc.cu)

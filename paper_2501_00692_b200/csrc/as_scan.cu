@@ -117,9 +117,9 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t limit = WAIT_LIMIT) {
   const uint32_t addr = smem_u32(bar);
-  for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+  for (uint32_t it = 0; it < limit; ++it) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -915,6 +915,20 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   if (fin) atomicAdd(db_delta + pmine, dbacc);
 }
 
+// Self test of the bounded wait: one warp waits for a phase of an mbarrier that nothing will ever complete, with a
+// short poll limit.  The wait must give up, the status word must read AS_ERR_TIMEOUT, and the kernel must return.
+__global__ void wait_selftest_kernel(int* status, uint32_t limit) {
+  __shared__ __align__(8) uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const bool ok = mbar_wait(&bar, 0, limit);
+  const int bad = __syncthreads_or(ok ? 0 : 1);
+  if (bad && threadIdx.x == 0) atomicExch(status, AS_ERR_TIMEOUT);
+}
+
 template <typename IO>
 __global__ void finish_dx_kernel(int64_t n, const float* __restrict__ acc, const IO* __restrict__ dxdir,
                                  IO* __restrict__ dx) {
@@ -1025,6 +1039,12 @@ int launch_adjoint_main(const Plan& pl, const ScanPtrs& sp, float* dA_log, float
                    : launch_main_t<__nv_bfloat16, false>(pl, sp, dA_log, db_delta, st);
   return pl.full ? launch_main_t<float, true>(pl, sp, dA_log, db_delta, st)
                  : launch_main_t<float, false>(pl, sp, dA_log, db_delta, st);
+}
+
+int launch_wait_selftest(int* status, unsigned limit, cudaStream_t st) {
+  wait_selftest_kernel<<<1, 32, 0, st>>>(status, limit);
+  count_launch();
+  return (int)cudaGetLastError();
 }
 
 int launch_finish_dx(const Plan& pl, const float* dxacc, const void* dxdir, void* dx, cudaStream_t st) {

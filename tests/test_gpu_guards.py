@@ -81,3 +81,22 @@ def test_no_write_outside_buffers(batch, T, P, tbar, io):
     B.as_rmsnorm_fwd(sh, x, y); B.as_rmsnorm_bwd_add(sh, x, dy, grads["dx"]); B.as_residual_add(sh, x, dy, y)
     check("glue")
     assert B.as_check_status(ws_v) == 0
+
+
+def test_bounded_wait_reports_timeout_and_context_survives():
+    """A device-side wait that can never be satisfied gives up after its poll limit, the host reads AS_ERR_TIMEOUT
+    from the status word, and the next call on the same context works and reports AS_OK."""
+    build_library()
+    ws = torch.zeros(4096, dtype=torch.uint8, device=DEV)
+    B.as_wait_selftest(ws, poll_limit=2048)
+    assert B.as_check_status(ws) == B.AS_ERR_TIMEOUT
+    w = synth.custom_workload("after", 19, 1, 64, 32, io="f32")
+    theta = synth.layer_params(w, 0, DEV)
+    x, _ = synth.activations(w, DEV)
+    sh = B.shape_of(x)
+    fb, _ = B.as_workspace_bytes(sh, 64)
+    ws2 = B.alloc_workspace(fb, DEV)
+    y = torch.empty_like(x)
+    B.as_ssm_forward(sh, theta, x, y, ws2)
+    assert B.as_check_status(ws2) == B.AS_OK
+    assert torch.isfinite(y).all()
