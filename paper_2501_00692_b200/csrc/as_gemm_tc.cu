@@ -1,6 +1,8 @@
 // bf16 tensor-core contractions for sm_100a: TMA (cp.async.bulk.tensor, 128-byte swizzle) feeds a
-// shared-memory ring, one elected thread issues tcgen05.mma into a TMEM accumulator, four warps drain it
-// with tcgen05.ld and apply the fused epilogue.  One kernel template covers the three token-dimension
+// shared-memory ring, one elected thread issues tcgen05.mma into a TMEM accumulator, eight warps drain it
+// with tcgen05.ld, apply the fused epilogue into a swizzled shared-memory staging tile and hand that tile to
+// TMA (bulk tensor store, or bulk tensor reduce-add for the split-K weight gradients), so that global memory
+// only sees whole rows of 64 bytes.  One kernel template covers the three token-dimension
 // contractions of the layer:
 //   PROJ : [Delta | B | C] = X Wcat^T            (A K-major, B K-major;  softplus+bias epilogue)
 //   DW   : dWcat = Gcat^T X  over all tokens     (A MN-major, B MN-major; split-K, fp32 reduction)
@@ -17,13 +19,14 @@ namespace {
 
 constexpr int BM = 128, BK = 64, UK = 16, EPI_WARPS = 8, NTHREADS = 64 + 32 * EPI_WARPS;
 constexpr int A_BYTES = BM * BK * 2;
+constexpr int EPI_TILE_BYTES = 32 * 64;   // staging tile of one epilogue warp: 32 rows of 64 bytes, 64-byte swizzle
 // tile width BN is a template parameter: 256 keeps the shared-memory operand traffic per MMA cycle under the
 // 128 B/clk an SM can read (a 128x128 tile needs 128 B/clk for the MMA alone), 128 wastes less on narrow outputs
 template <int BN> struct Cfg {
   static constexpr int B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES = BN >= 208 ? 4 : 6;
   static constexpr int TMEM_COLS = 2 * BN <= 256 ? 256 : 512;   // two accumulators, power-of-two allocation
-  static constexpr int SMEM_DYN = STAGES * STAGE_BYTES + 1024;   // + slack for 1024-byte alignment
+  static constexpr int SMEM_DYN = STAGES * STAGE_BYTES + 1024 + EPI_WARPS * 2 * EPI_TILE_BYTES;   // + alignment slack + staging
 };
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
@@ -36,12 +39,7 @@ struct TcArgs {
   int kblocks;          // number of BK-blocks along K
   int splitk;
   int P;                // d_model
-  // PROJ
-  float* delta; float* bc; const float* bias;
-  // DW
-  float* dW_delta; float* dW_B; float* dW_C;
-  // DX
-  const __nv_bfloat16* dxdir; __nv_bfloat16* dx;
+  const float* bias;    // PROJ: b_delta
   int* status;
 };
 
@@ -131,6 +129,24 @@ __device__ __forceinline__ float softplus_f(float u) {
   return fmaxf(u, 0.f) + (z < 0.0078125f ? small : big);
 }
 
+// ---- TMA stores out of the staging tile (bulk async-groups are tracked per issuing thread) ----
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, const void* src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(tm), "r"(c0), "r"(c1), "r"(smem_u32(src)) : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* tm, const void* src, int c0, int c1) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(tm), "r"(c0), "r"(c1), "r"(smem_u32(src)) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// byte offset of 16-byte piece q of row r in a [rows][64 B] tile under the 64-byte swizzle
+__device__ __forceinline__ uint32_t swz64(int r, int q) { return (uint32_t)(r * 64 + ((q ^ ((r >> 1) & 3)) << 4)); }
+
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -143,13 +159,17 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 // Tile order: n fastest, then m, then the K split, so concurrently running CTAs share A rows through L2.
 template <int AMAJ, int BMAJ, int EPI, int BN>
 __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
-                                                           const __grid_constant__ CUtensorMap tmB, TcArgs a) {
+                                                           const __grid_constant__ CUtensorMap tmB,
+                                                           const __grid_constant__ CUtensorMap tmO0,
+                                                           const __grid_constant__ CUtensorMap tmO1,
+                                                           const __grid_constant__ CUtensorMap tmO2, TcArgs a) {
   constexpr int STAGES = Cfg<BN>::STAGES, B_BYTES = Cfg<BN>::B_BYTES, STAGE_BYTES = Cfg<BN>::STAGE_BYTES;
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[STAGES];
   __shared__ __align__(8) uint64_t empty_bar[STAGES];
   __shared__ __align__(8) uint64_t tmem_full_bar[2];
   __shared__ __align__(8) uint64_t tmem_empty_bar[2];
+  __shared__ __align__(8) uint64_t ld_bar[EPI_WARPS][2];   // DX: arrival of the dx_dir tile in a staging buffer
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
 
@@ -163,6 +183,7 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full_bar[b], 1); mbar_init(&tmem_empty_bar[b], EPI_WARPS); }
+    for (int w2 = 0; w2 < EPI_WARPS; ++w2) { mbar_init(&ld_bar[w2][0], 1); mbar_init(&ld_bar[w2][1], 1); }
     abort_s = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -256,56 +277,58 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
     }
   } else {
     // ---------------- epilogue warps ----------------
+    // A warp owns TMEM lanes [32 quarter, 32 quarter + 32) = 32 output rows, one row per lane, and walks its share of
+    // the tile's columns in chunks that are 64 bytes wide in the output (16 fp32 or 32 bf16 columns).  A chunk goes
+    // registers -> staging tile (two per warp, alternating) -> TMA; lane 0 issues and tracks the bulk operations.
+    // Rows and columns past the output's extent are clipped by TMA.
     const int quarter = warp & 3;              // the TMEM lane quarter this warp may read
     const int chalf = (warp - 2) / 4;          // which half of the tile's columns it drains
-    constexpr int NCHUNK = BN / 16;                            // 16-column chunks of a tile
+    constexpr int CW = EPI == TC_DX ? 32 : 16;                 // columns per chunk
+    constexpr int NCHUNK = BN / CW;
     constexpr int CSPLIT = (NCHUNK + 1) / 2;                   // first warp of a quarter takes [0, CSPLIT)
+    uint8_t* stg = smem + STAGES * STAGE_BYTES + (warp - 2) * 2 * EPI_TILE_BYTES;
+    uint64_t* lbar = ld_bar[warp - 2];
+    const int c_lo = chalf ? CSPLIT : 0, c_hi = chalf ? NCHUNK : CSPLIT;
     int ti = 0;
+    uint32_t nchunks_done = 0;                 // chunks this warp has staged so far (selects buffer and mbarrier phase)
     bool ok = true;
     for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++ti) {
       int64_t m0; int n0, kb0, nkb;
       decode(t, m0, n0, kb0, nkb);
       const int ab = ti & 1, around = ti >> 1;
       if (nkb > 0) {
+        const int mrow = (int)m0 + quarter * 32;      // first output row of this warp
+        if (EPI == TC_DX && lane == 0 && n0 + c_lo * CW < a.N) {
+          // dx_dir tile of the first chunk; later ones are requested one chunk ahead
+          bulk_wait_read<0>();
+          const uint32_t bi = nchunks_done & 1;
+          mbar_expect_tx(&lbar[bi], EPI_TILE_BYTES);
+          tma_load_2d(stg + bi * EPI_TILE_BYTES, &tmO1, n0 + c_lo * CW, mrow, &lbar[bi]);
+        }
         if (!mbar_wait(&tmem_full_bar[ab], around & 1, abortp)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const int64_t m = m0 + quarter * 32 + lane;   // this thread's output row
 #pragma unroll 1
-        for (int c = chalf ? CSPLIT : 0; c < (chalf ? NCHUNK : CSPLIT); ++c) {
-          uint32_t r[16];
-          tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(ab * BN + c * 16), r);
-          const int nb = n0 + c * 16;
-          if (m >= a.M || nb >= a.N) continue;
-          if (EPI == TC_PROJ) {
-            if (nb < a.P) {
-              float4* dst = reinterpret_cast<float4*>(a.delta + m * a.P + nb);
-              const float4* b4 = reinterpret_cast<const float4*>(a.bias + nb);
-#pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                const float4 bv = __ldg(b4 + q);
-                dst[q] = make_float4(softplus_f(__uint_as_float(r[4 * q]) + bv.x), softplus_f(__uint_as_float(r[4 * q + 1]) + bv.y),
-                                     softplus_f(__uint_as_float(r[4 * q + 2]) + bv.z), softplus_f(__uint_as_float(r[4 * q + 3]) + bv.w));
+        for (int c = c_lo; c < c_hi; ++c) {
+          const int nb = n0 + c * CW;
+          if (nb >= a.N) break;                        // warp-uniform
+          const uint32_t bi = nchunks_done & 1;
+          uint8_t* buf = stg + bi * EPI_TILE_BYTES;
+          const uint32_t tcol = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(ab * BN + c * CW);
+          if (EPI == TC_DX) {
+            if (lane == 0) {
+              bulk_wait_read<0>();                      // the other buffer's store has been read out
+              if (c + 1 < c_hi && nb + CW < a.N) {
+                mbar_expect_tx(&lbar[bi ^ 1], EPI_TILE_BYTES);
+                tma_load_2d(stg + (bi ^ 1) * EPI_TILE_BYTES, &tmO1, nb + CW, mrow, &lbar[bi ^ 1]);
               }
-            } else {
-              float4* dst = reinterpret_cast<float4*>(a.bc + m * NBC + (nb - a.P));
-#pragma unroll
-              for (int q = 0; q < 4; ++q)
-                dst[q] = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]), __uint_as_float(r[4 * q + 2]),
-                                     __uint_as_float(r[4 * q + 3]));
             }
-          } else if (EPI == TC_DW) {
-            float* dst;
-            if (m < a.P) dst = a.dW_delta + m * a.P + nb;
-            else if (m < a.P + NS) dst = a.dW_B + (m - a.P) * a.P + nb;
-            else dst = a.dW_C + (m - a.P - NS) * a.P + nb;
+            uint32_t r[32];
+            tmem_ld32(tcol, r);
+            if (!mbar_wait(&lbar[bi], (nchunks_done >> 1) & 1, abortp)) { ok = false; break; }
 #pragma unroll
-            for (int j = 0; j < 16; ++j) atomicAdd(dst + j, __uint_as_float(r[j]));
-          } else {
-            const uint4* src = reinterpret_cast<const uint4*>(a.dxdir + m * a.P + nb);
-            uint4* dst = reinterpret_cast<uint4*>(a.dx + m * a.P + nb);
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
-              const uint4 sv = __ldg(src + q);
+            for (int q = 0; q < 4; ++q) {
+              uint4* pq = reinterpret_cast<uint4*>(buf + swz64(lane, q));
+              const uint4 sv = *pq;
               const __nv_bfloat162* s2 = reinterpret_cast<const __nv_bfloat162*>(&sv);
               uint4 ov;
               __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
@@ -314,16 +337,60 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
                 const float2 f = __bfloat1622float2(s2[e]);
                 o2[e] = __floats2bfloat162_rn(f.x + __uint_as_float(r[8 * q + 2 * e]), f.y + __uint_as_float(r[8 * q + 2 * e + 1]));
               }
-              dst[q] = ov;
+              *pq = ov;
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) { tma_store_2d(&tmO0, buf, nb, mrow); bulk_commit(); }
+          } else {
+            uint32_t r[16];
+            tmem_ld16(tcol, r);
+            if (lane == 0) bulk_wait_read<1>();         // the operation that last used this buffer has read it
+            __syncwarp();
+            if (EPI == TC_PROJ && nb < a.P) {
+              const float4* b4 = reinterpret_cast<const float4*>(a.bias + nb);
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const float4 bv = __ldg(b4 + q);
+                *reinterpret_cast<float4*>(buf + swz64(lane, q)) =
+                    make_float4(softplus_f(__uint_as_float(r[4 * q]) + bv.x), softplus_f(__uint_as_float(r[4 * q + 1]) + bv.y),
+                                softplus_f(__uint_as_float(r[4 * q + 2]) + bv.z), softplus_f(__uint_as_float(r[4 * q + 3]) + bv.w));
+              }
+            } else {
+#pragma unroll
+              for (int q = 0; q < 4; ++q)
+                *reinterpret_cast<uint4*>(buf + swz64(lane, q)) = make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              if (EPI == TC_PROJ) {
+                if (nb < a.P) tma_store_2d(&tmO0, buf, nb, mrow);       // Delta
+                else tma_store_2d(&tmO1, buf, nb - a.P, mrow);          // [B | C]
+              } else {
+                // rows of Wcat space: [0, P) dW_delta, [P, P+16) dW_B, [P+16, P+32) dW_C; 16-row groups never straddle
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                  const int mr = mrow + 16 * hh;
+                  const void* src = buf + hh * 1024;
+                  if (mr < a.P) tma_reduce_add_2d(&tmO0, src, nb, mr);
+                  else if (mr < a.P + NS) tma_reduce_add_2d(&tmO1, src, nb, mr - a.P);
+                  else if (mr < a.P + 2 * NS) tma_reduce_add_2d(&tmO2, src, nb, mr - a.P - NS);
+                }
+              }
+              bulk_commit();
             }
           }
+          ++nchunks_done;
         }
+        if (!ok) break;
         // hand the accumulator buffer back to the issuer
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncwarp();
         if (lane == 0) mbar_arrive(&tmem_empty_bar[ab]);
       }
     }
+    if (lane == 0) bulk_wait_all();            // staging tiles must outlive the bulk operations that read them
     if (!ok) { *abortp = 1; if (lane == 0) atomicExch(a.status, AS_ERR_TIMEOUT); }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -367,22 +434,33 @@ EncodeTiledFn get_encode() {
   return fn;
 }
 
-// bf16 row-major [rows, cols] with row pitch `ld` elements; box = {64 cols, box_rows}; 128-byte swizzle; OOB reads 0
-int make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows) {
+// row-major [rows, cols] tensor with row pitch `ld` elements; box = {box_cols, box_rows}; OOB reads give 0, OOB writes are dropped
+int make_map_t(CUtensorMap* tm, CUtensorMapDataType dt, int esz, CUtensorMapSwizzle swz, const void* base, uint64_t rows,
+               uint64_t cols, uint64_t ld, uint32_t box_cols, uint32_t box_rows) {
   EncodeTiledFn enc = get_encode();
   if (!enc) return 1;
   cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {ld * 2};
-  cuuint32_t box[2] = {64, box_rows};
+  cuuint64_t strides[1] = {ld * (uint64_t)esz};
+  cuuint32_t box[2] = {box_cols, box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r = enc(tm, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? 0 : 1;
+}
+// bf16 operand: box = {64 cols, box_rows}, 128-byte swizzle
+int make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows) {
+  return make_map_t(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, CU_TENSOR_MAP_SWIZZLE_128B, base, rows, cols, ld, 64, box_rows);
+}
+// epilogue tiles: rows of 64 bytes, 64-byte swizzle
+int make_map_out_f32(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  return make_map_t(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, CU_TENSOR_MAP_SWIZZLE_64B, base, rows, cols, cols, 16, box_rows);
+}
+int make_map_out_bf16(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols) {
+  return make_map_t(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, CU_TENSOR_MAP_SWIZZLE_64B, base, rows, cols, cols, 32, 32);
 }
 
 template <int AMAJ, int BMAJ, int EPI, int BN>
-int launch_tc(const CUtensorMap& tmA, const CUtensorMap& tmB, const TcArgs& a, cudaStream_t st) {
+int launch_tc(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap (&tmO)[3], const TcArgs& a, cudaStream_t st) {
   static bool attr_set = false;
   auto kern = gemm_tc_kernel<AMAJ, BMAJ, EPI, BN>;
   if (!attr_set) {
@@ -391,7 +469,7 @@ int launch_tc(const CUtensorMap& tmA, const CUtensorMap& tmB, const TcArgs& a, c
   }
   const int64_t ntiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN) * a.splitk;
   const unsigned grid = (unsigned)(ntiles < 148 ? ntiles : 148);   // one persistent CTA per SM
-  kern<<<grid, NTHREADS, Cfg<BN>::SMEM_DYN, st>>>(tmA, tmB, a);
+  kern<<<grid, NTHREADS, Cfg<BN>::SMEM_DYN, st>>>(tmA, tmB, tmO[0], tmO[1], tmO[2], a);
   count_launch();
   return (int)cudaGetLastError();
 }
@@ -418,9 +496,13 @@ int tc_projections(const Plan& pl, const as_params_t* pr, const void* x, char* w
   if (make_map(&tmB, ws + pl.off_wcat, NW, P, P, PBN)) return 1;
   TcArgs a{};
   a.M = M; a.N = NW; a.kblocks = (P + BK - 1) / BK; a.splitk = 1; a.P = P;
-  a.delta = (float*)(ws + pl.off_delta); a.bc = (float*)(ws + pl.off_bc); a.bias = pr->b_delta;
+  a.bias = pr->b_delta;
   a.status = (int*)(ws + pl.off_status);
-  return launch_tc<MAJ_K, MAJ_K, TC_PROJ, PBN>(tmA, tmB, a, st);
+  CUtensorMap tmO[3];
+  if (make_map_out_f32(&tmO[0], ws + pl.off_delta, M, P, 32)) return 1;
+  if (make_map_out_f32(&tmO[1], ws + pl.off_bc, M, NBC, 32)) return 1;
+  tmO[2] = tmO[1];
+  return launch_tc<MAJ_K, MAJ_K, TC_PROJ, PBN>(tmA, tmB, tmO, a, st);
 }
 
 int tc_weight_grads(const Plan& pl, const void* x, const as_grads_t* out, char* ws, cudaStream_t st) {
@@ -441,9 +523,12 @@ int tc_weight_grads(const Plan& pl, const void* x, const as_grads_t* out, char* 
   if (sk < 1) sk = 1;
   const int kper = (a.kblocks + sk - 1) / sk;
   a.splitk = (a.kblocks + kper - 1) / kper;   // no empty split: every tile has at least one K block
-  a.dW_delta = out->dW_delta; a.dW_B = out->dW_B; a.dW_C = out->dW_C;
   a.status = (int*)(ws + pl.off_status);
-  return launch_tc<MAJ_MN, MAJ_MN, TC_DW, TBN>(tmA, tmB, a, st);
+  CUtensorMap tmO[3];
+  if (make_map_out_f32(&tmO[0], out->dW_delta, P, P, 16)) return 1;
+  if (make_map_out_f32(&tmO[1], out->dW_B, NS, P, 16)) return 1;
+  if (make_map_out_f32(&tmO[2], out->dW_C, NS, P, 16)) return 1;
+  return launch_tc<MAJ_MN, MAJ_MN, TC_DW, TBN>(tmA, tmB, tmO, a, st);
 }
 
 int tc_input_grad(const Plan& pl, void* dx, char* ws, cudaStream_t st) {
@@ -454,9 +539,12 @@ int tc_input_grad(const Plan& pl, void* dx, char* ws, cudaStream_t st) {
   if (make_map(&tmB, ws + pl.off_wcat, NW, P, P, 64)) return 1;      // Wcat as [K=P+32, N=P]
   TcArgs a{};
   a.M = M; a.N = P; a.kblocks = (NW + BK - 1) / BK; a.splitk = 1; a.P = P;
-  a.dxdir = (const __nv_bfloat16*)(ws + pl.off_dxdir); a.dx = (__nv_bfloat16*)dx;
   a.status = (int*)(ws + pl.off_status);
-  return launch_tc<MAJ_K, MAJ_MN, TC_DX, TBN>(tmA, tmB, a, st);
+  CUtensorMap tmO[3];
+  if (make_map_out_bf16(&tmO[0], dx, M, P)) return 1;
+  if (make_map_out_bf16(&tmO[1], ws + pl.off_dxdir, M, P)) return 1;
+  tmO[2] = tmO[1];
+  return launch_tc<MAJ_K, MAJ_MN, TC_DX, TBN>(tmA, tmB, tmO, a, st);
 }
 
 }  // namespace as
