@@ -9,7 +9,9 @@
 // Arithmetic on the two states (2m, 2m+1) of a channel is packed into f32x2 instructions, which halves
 // the issue slots the FP32 pipe needs and leaves room for MUFU.EX2, shuffles and shared-memory loads.
 // Inputs of a chunk (x, Delta, dy tiles by 2D TMA; B/C rows, the chunk checkpoint and its cumulative
-// Delta by 1D bulk copies) land in a 3-stage shared-memory ring guarded by mbarriers with bounded waits.
+// Delta by 1D bulk copies) land in a shared-memory ring guarded by mbarriers with bounded waits.  The main
+// adjoint kernel parks the rebuilt per-token states of a chunk in tensor memory (tcgen05.st / tcgen05.ld)
+// instead of registers or shared memory.
 #include <cuda.h>
 
 #include "as_internal.cuh"
@@ -32,7 +34,7 @@ int make_plan(const as_shape_t* sh, int64_t tbar, Plan* pl) {
   p.bw = p.P < CH ? p.P : CH;
   const int64_t ctas = (int64_t)p.tiles * p.B;
   // two full waves of the main kernel's resident CTAs (148 SMs x CTAs per SM), never more than that
-  const int64_t slots = 148 * (NCH == 2 ? 3 : 4);
+  const int64_t slots = 148 * 3;
   int64_t s_target = (2 * slots) / ctas;
   if (s_target < 1) s_target = 1;
   int64_t L = (p.T + s_target - 1) / s_target;
@@ -158,8 +160,8 @@ struct Stage {
 };
 constexpr int NSTAGE = 3;        // ascending kernels
 constexpr int WRED_Q = 32 * 4 + 8;   // floats per quarter-block of the per-warp reduction scratch (512 B + 32 B skew)
-constexpr int MAIN_CTAS = NCH == 2 ? 3 : 4;   // resident CTAs per SM the main kernel is compiled for
-constexpr int HALF = CK / 2;       // tokens per unrolled loop body of the main adjoint kernel
+constexpr int MAIN_CTAS = 3;    // resident CTAs per SM the main kernel is compiled for (168 registers per thread)
+constexpr int HALF = CK / 2;       // unroll factor of the main adjoint kernel's backward token loop
 constexpr int NSTAGE_MAIN = 2;   // main adjoint kernel: a chunk takes thousands of cycles, one chunk of lookahead suffices
 
 // per-thread values of its NCH channels
@@ -551,20 +553,100 @@ __global__ void __launch_bounds__(NTHR) fixup_mu_kernel(Plan pl, const float* __
 //       mu_i = gC_i + abar_{i+1} mu_{i+1} - W_i gC_{i+Tbar}
 //   and evaluating the per-token VJPs.
 // ------------------------------------------------------------------------------------------------
+template <bool B> struct BoolC { static constexpr bool v = B; };
+// ---- tensor memory as a per-thread scratchpad ------------------------------------------------------
+// The main adjoint kernel runs no MMA, so the SM's tensor memory is free.  Each CTA allocates 128 of the 512
+// columns of its SM (three CTAs are resident) and every thread parks per-token states in its own TMEM lane:
+// warp w of the 4-warp CTA owns lanes [32w, 32w+32), a 32x32b access moves 16 registers of each lane to or
+// from 16 consecutive columns.
+constexpr int TM_COLS = 128;
+constexpr int TM_HST = 7 * 16;   // columns [16 j, 16 j + 16): state after token j (j = 0..6); [112, 128): segment-start state
+
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const u64 (&v)[NU]) {
+  uint32_t r[16];
+#pragma unroll
+  for (int u = 0; u < 8; ++u) asm("mov.b64 {%0, %1}, %2;" : "=r"(r[2 * u]), "=r"(r[2 * u + 1]) : "l"(v[u]));
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, u64 (&v)[NU]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int u = 0; u < 8; ++u) asm("mov.b64 %0, {%1, %2};" : "=l"(v[u]) : "r"(r[2 * u]), "r"(r[2 * u + 1]));
+}
+// split form: the load is issued early and its registers are only read after tmem_ld16_wait, which names them as
+// read-write operands so that the compiler cannot move a use (or a copy) of them above the wait
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld16_wait(uint32_t (&r)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+                 "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+               :
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// shared-memory stage of one chunk of the main adjoint kernel (the chunk checkpoint has a buffer of its own)
+template <int ESZ, bool WIN>
+struct StageM {
+  static constexpr int X = 0;
+  static constexpr int D = X + CK * CH * ESZ;
+  static constexpr int BC = D + CK * CH * 4;
+  static constexpr int G = BC + CK * NBC * 4;
+  static constexpr int CS = G + CK * CH * ESZ;
+  static constexpr int G2 = CS + CH * 4;
+  static constexpr int D2 = G2 + (WIN ? CK * CH * ESZ : 0);
+  static constexpr int BC2 = D2 + (WIN ? CK * CH * 4 : 0);
+  static constexpr int BYTES = BC2 + (WIN ? CK * NBC * 4 : 0);
+};
+template <int ESZ, bool WIN> struct MainCfg {
+  static constexpr int SMEM_DYN = NSTAGE_MAIN * StageM<ESZ, WIN>::BYTES + TILE_FLOATS * 4 + 128;
+};
+
+// ------------------------------------------------------------------------------------------------
+// main adjoint kernel: one CTA per (channel tile, segment, batch element), chunks walked last to first.
+// Per chunk: rebuild the states after tokens 0..6 from the chunk checkpoint and park them in tensor memory,
+// then walk the chunk's tokens backwards: mu recurrence (with the exact window exit), the per-token
+// vector-Jacobian products, the channel sums dB_t / dC_t, and the per-channel outputs du_t and dx_dir_t.
+// ------------------------------------------------------------------------------------------------
 template <typename IO, bool FULL>
 __global__ void __launch_bounds__(NTHR, MAIN_CTAS)
 adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmD,
                     const __grid_constant__ CUtensorMap tmG, Plan pl, const float* __restrict__ A_log,
                     char* __restrict__ ws, float* __restrict__ dA_log, float* __restrict__ db_delta) {
+  static_assert(NCH == 2 && NTHR == 128, "tensor-memory parking assumes 4 warps and 16 state registers per thread");
   constexpr int ESZ = IoSz<IO>::v;
   constexpr bool WIN = !FULL;
-  using St = Stage<ESZ, true, true, WIN>;
+  using St = StageM<ESZ, WIN>;
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[NSTAGE_MAIN];
+  __shared__ __align__(8) uint64_t ckp_bar;          // the checkpoint tile of the current chunk has landed
+  __shared__ __align__(8) uint64_t ckp_free;         // all threads have read it (NTHR arrivals)
+  __shared__ uint32_t tmem_base_s;
   __shared__ float red[2][CK][NBC];                 // per-token [dB | dC] sums of the CTA, two chunks in flight
   __shared__ __align__(16) float wred[NTHR / 32][4 * WRED_Q];   // per-warp scratch of the channel reduction
-  __shared__ ulonglong2 hst_s[2 * NCH][NTHR];
   uint8_t* smem = smem_raw + ((128u - (smem_u32(smem_raw) & 127u)) & 127u);   // stays a shared-space pointer
+  uint8_t* ckp_s = smem + NSTAGE_MAIN * St::BYTES;
 
   const int tile = blockIdx.x, s = blockIdx.y, b = blockIdx.z;
   const int P = pl.P;
@@ -582,21 +664,30 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   const int ncs = min(CH, P - tile * CH);   // channels of this tile that exist
   const int64_t BT = (int64_t)pl.B * T;
   const int du_ld = pl.du_ld;
-  // the two lanes of a pair end up with the same per-channel sums: with two channels per thread lane `half`
-  // finalises channel `half`, with one channel per thread lane 0 does
-  const int chf = NCH == 2 ? w.half : 0;
-  const bool fin = w.act && (NCH == 2 || w.half == 0);
+  // the two lanes of a pair end up with the same per-channel sums: lane `half` finalises channel `half`
+  const int chf = w.half;
+  const bool fin = w.act;
   const int pmine = w.pa + chf;
   IO* du = reinterpret_cast<IO*>(ws + pl.off_du) + pmine;
   IO* dxdir = reinterpret_cast<IO*>(ws + pl.off_dxdir) + pmine;
 
   if (w.tid == 0) {
     for (int i = 0; i < NSTAGE_MAIN; ++i) mbar_init(&full_bar[i], 1);
+    mbar_init(&ckp_bar, 1);
+    mbar_init(&ckp_free, NTHR);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "n"(TM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
   for (int e = w.tid; e < 2 * CK * NBC; e += NTHR) (&red[0][0][0])[e] = 0.f;
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  const uint32_t tx_base = (uint32_t)(CK * CH * ESZ * 2 + CK * CH * 4 + CK * NBC * 4 + TILE_FLOATS * 4 + ncs * 4 +
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tm = tmem_base_s + ((uint32_t)(32 * warp) << 16);   // this warp's lanes, column 0 of the allocation
+  const uint32_t tx_base = (uint32_t)(CK * CH * ESZ * 2 + CK * CH * 4 + CK * NBC * 4 + ncs * 4 +
                                       (WIN ? CK * CH * ESZ + CK * CH * 4 : 0));
   // chunks are visited last to first: the i-th visited chunk is c = nchunk-1-i
   auto issue = [&](int i) {
@@ -613,7 +704,6 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     tma_2d(sm + St::D, &tmD, tile * CH, row, &full_bar[st]);
     tma_2d(sm + St::G, &tmG, tile * CH, row, &full_bar[st]);
     bulk_1d(sm + St::BC, bc + row * NBC, CK * NBC * 4, &full_bar[st]);
-    bulk_1d(sm + St::CKP, ckpt + (cc * pl.tiles + tile) * TILE_FLOATS, TILE_FLOATS * 4, &full_bar[st]);
     bulk_1d(sm + St::CS, cs + cc * P + tile * CH, ncs * 4, &full_bar[st]);
     if (WIN) {
       // rows of the tokens leaving the window; past the end of the whole tensor TMA fills zeros, and rows
@@ -623,18 +713,26 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
       if (win_rows) bulk_1d(sm + St::BC2, bc + row2 * NBC, CK * NBC * 4, &full_bar[st]);
     }
   };
-  if (w.tid == 0)
+  auto issue_ckp = [&](int i) {   // checkpoint tile of the i-th visited chunk (single buffer)
+    const int c = nchunk - 1 - i;
+    const int64_t cc = (int64_t)b * pl.NC + (t0 + (int64_t)c * CK) / CK;
+    mbar_expect_tx(&ckp_bar, TILE_FLOATS * 4);
+    bulk_1d(ckp_s, ckpt + (cc * pl.tiles + tile) * TILE_FLOATS, TILE_FLOATS * 4, &ckp_bar);
+  };
+  if (w.tid == 0) {
     for (int i = 0; i < NSTAGE_MAIN && i < nchunk; ++i) issue(i);
+    issue_ckp(0);
+  }
 
   u64 A2[NU], mu[NU], dAacc[NU];
   load_A2(A_log, w, A2);
   const int64_t sb = ((int64_t)b * pl.S + s) * pl.tiles + tile;
   load_block_g(reinterpret_cast<const float*>(ws + pl.off_carry) + sb * TILE_FLOATS, w.tid, mu);
-  {   // true segment-start state: parked in shared memory, read back once per chunk
+  {   // true segment-start state: parked in tensor memory, read back once per chunk
     u64 hst[NU];
     load_block_g(reinterpret_cast<const float*>(ws + pl.off_hstart) + sb * TILE_FLOATS, w.tid, hst);
-#pragma unroll
-    for (int q = 0; q < 2 * NCH; ++q) hst_s[q][w.tid] = make_ulonglong2(hst[2 * q], hst[2 * q + 1]);
+    tmem_st16(tm + TM_HST, hst);
+    tmem_wait_st();
   }
 #pragma unroll
   for (int u = 0; u < NU; ++u) dAacc[u] = 0ull;
@@ -656,12 +754,15 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     for (int c = 0; c < NCH; ++c) sw[c] = swp[c];
   }
   float dbacc = 0.f;
+  bool failed = false;
 
   for (int i = 0; i < nchunk; ++i) {
     const int st = i % NSTAGE_MAIN;
     const int c = nchunk - 1 - i;
     uint8_t* sm = smem + st * St::BYTES;
-    const bool ok = mbar_wait(&full_bar[st], (i / NSTAGE_MAIN) & 1);
+    bool ok = mbar_wait(&full_bar[st], (i / NSTAGE_MAIN) & 1);
+    ok = mbar_wait(&ckp_bar, i & 1) && ok;
+    ok = __all_sync(0xffffffffu, ok);   // warp-uniform: the tensor-memory accesses below are warp-collective
     const int64_t tc = t0 + (int64_t)c * CK;
     const int nt = (int)min((int64_t)CK, t1 - tc);
     const int rb = i & 1;
@@ -671,6 +772,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
 #pragma unroll
     for (int c = 0; c < NCH; ++c) { swc[c] = (float)sw[c]; swl[c] = 0.f; dsumc[c] = 0.f; sd2[c] = 0.f; }
     bool chunk_live = false;   // warp-uniform: does any exit factor W of this chunk reach 2^-64 ?
+    bool tfail = false;
     if (nt < CK) {   // only the last chunk of a sequence: neutralise the slots past its end
       if (ok) {
         zero_rows(sm + St::D, CH * 4, nt, w.tid);
@@ -682,9 +784,11 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     if (ok) {
       // state at the chunk start: local checkpoint + decayed true segment-start state
       u64 h[NU];
-      load_block(reinterpret_cast<const float*>(sm + St::CKP), w.tid, h);
+      load_block(reinterpret_cast<const float*>(ckp_s), w.tid, h);
+      mbar_arrive(&ckp_free);   // this thread is done with the checkpoint buffer
       {
-        u64 c2[NCH];
+        u64 hst[NU], c2[NCH];
+        tmem_ld16(tm + TM_HST, hst);
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
           float csv = *reinterpret_cast<const float*>(sm + St::CS + 4 * (NCH * w.k + c));
@@ -692,11 +796,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
           c2[c] = pk(csv, csv);
         }
 #pragma unroll
-        for (int q = 0; q < 2 * NCH; ++q) {
-          const ulonglong2 hq = hst_s[q][w.tid];
-          h[2 * q] = fma2(ex2_2(mul2(c2[q / 2], A2[2 * q])), hq.x, h[2 * q]);
-          h[2 * q + 1] = fma2(ex2_2(mul2(c2[q / 2], A2[2 * q + 1])), hq.y, h[2 * q + 1]);
-        }
+        for (int u = 0; u < NU; ++u) h[u] = fma2(ex2_2(mul2(c2[u / 4], A2[u])), hst[u], h[u]);
       }
       if (WIN) {
         // Delta of the tokens leaving the window during this chunk.  Inside the chunk the window sum never drops
@@ -714,22 +814,14 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         for (int c = 0; c < NCH; ++c) live = live || ((swc[c] - sd2[c]) * a2max[c] > -64.f);
         chunk_live = __any_sync(0xffffffffu, live && w.act && nwin > 0);
       }
-      // forward rebuild in two halves of four tokens (one copy of the code, rolled loop): only the states
-      // after tokens 0, 2, 4, 6 are kept; `cur` holds the pair of the half being processed, `hsA` parks the
-      // first half's pair while the second half is rebuilt and walked.
-      u64 hsA[2][NU], cur[2][NU];
+      // forward rebuild: the states after tokens 0..6 go to tensor memory; the one after token 6 also stays in h
+      {
+        const float* bck = reinterpret_cast<const float*>(sm + St::BC) + 8 * w.half;
 #pragma unroll 1
-      for (int k = 0; k < 2; ++k) {
-        const uint8_t* smk = sm + k * HALF * CH * ESZ;          // x rows of this half
-        const uint8_t* smd = sm + St::D + k * HALF * CH * 4;
-        const float* bck = reinterpret_cast<const float*>(sm + St::BC) + k * HALF * NBC + 8 * w.half;
-#pragma unroll
-        for (int jj = 0; jj < HALF; ++jj) {
-          if (jj == HALF - 1 && k == 1) break;                  // the state after the chunk's last token is rebuilt below
-          __syncwarp();   // keeps the staged loads of later tokens from being hoisted (register pressure)
-          const ChV dv = lds_ch<float>(smd, jj, w.k);
-          const ChV xv = lds_ch<IO>(smk + St::X, jj, w.k);
-          const float* brow = bck + jj * NBC;
+        for (int j = 0; j < CK - 1; ++j) {
+          const ChV dv = lds_ch<float>(sm + St::D, j, w.k);
+          const ChV xv = lds_ch<IO>(sm + St::X, j, w.k);
+          const float* brow = bck + j * NBC;
           const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
           const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
           const u64 Bp[4] = {b01.x, b01.y, b23.x, b23.y};
@@ -741,81 +833,75 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
           }
 #pragma unroll
           for (int u = 0; u < NU; ++u) h[u] = fma2(ex2_2(mul2(d2[u / 4], A2[u])), h[u], mul2(dx2[u / 4], Bp[u % 4]));
-          if ((jj & 1) == 0) {
-#pragma unroll
-            for (int u = 0; u < NU; ++u) cur[jj / 2][u] = h[u];
-          }
+          tmem_st16(tm + 16 * j, h);
         }
-        if (k == 0) {
-#pragma unroll
-          for (int u = 0; u < NU; ++u) { hsA[0][u] = cur[0][u]; hsA[1][u] = cur[1][u]; }
-        }
+        tmem_wait_st();
+      }
+      if (w.tid == 0 && i + 1 < nchunk) {
+        // every thread has copied the checkpoint into registers long ago: fetch the next chunk's
+        if (mbar_wait(&ckp_free, i & 1)) issue_ckp(i + 1);
+        else tfail = true;
       }
       // output rows of this chunk, walked from its last token down
       IO* du_p = du + ((int64_t)b * T + tc + (CK - 1)) * du_ld;
       IO* dx_p = dxdir + ((int64_t)b * T + tc + (CK - 1)) * P;
-      // backward walk, second half first
-#pragma unroll 1
-      for (int k = 1; k >= 0; --k) {
-        if (k == 0) {
+      const float* bck = reinterpret_cast<const float*>(sm + St::BC) + 8 * w.half;
+      // backward walk.  Token 7's state is rebuilt from the state after token 6 (still in h); the others come back
+      // from tensor memory.  abar_i h_{i-1} is formed as h_i - Delta_i x_i B_i.
+#pragma unroll HALF
+      for (int j = CK - 1; j >= 0; --j) {
+        u64 hT[NU];
+        if (j < CK - 1) tmem_ld16(tm + 16 * j, hT);
+        const ChV dv = lds_ch<float>(sm + St::D, j, w.k);
+        const ChV xv = lds_ch<IO>(sm + St::X, j, w.k);
+        const ChV gv = lds_ch<IO>(sm + St::G, j, w.k);
+        const float* brow = bck + j * NBC;
+        const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
+        const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
+        const ulonglong2 c01 = *reinterpret_cast<const ulonglong2*>(brow + NS);
+        const ulonglong2 c23 = *reinterpret_cast<const ulonglong2*>(brow + NS + 4);
+        const u64 Bp[4] = {b01.x, b01.y, b23.x, b23.y};
+        const u64 Cp[4] = {c01.x, c01.y, c23.x, c23.y};
+        float dd[NCH], xs[NCH];
+        u64 d2[NCH], dx2[NCH], g2[NCH];
 #pragma unroll
-          for (int u = 0; u < NU; ++u) { cur[0][u] = hsA[0][u]; cur[1][u] = hsA[1][u]; }
+        for (int c = 0; c < NCH; ++c) {
+          dd[c] = dv.v[c]; xs[c] = xv.v[c];
+          const float dxc = dv.v[c] * xv.v[c];
+          d2[c] = pk(dd[c], dd[c]); dx2[c] = pk(dxc, dxc); g2[c] = pk(gv.v[c], gv.v[c]);
         }
-        const uint8_t* smk = sm + k * HALF * CH * ESZ;          // x / dy rows of this half
-        const uint8_t* smd = sm + k * HALF * CH * 4;            // Delta rows
-        const float* bck = reinterpret_cast<const float*>(sm) + k * HALF * NBC + 8 * w.half;
+        // mu_i += g_i C_i   (mu already carries abar_{i+1} mu_{i+1})
 #pragma unroll
-        for (int jj = HALF - 1; jj >= 0; --jj) {
-          const int j = k * HALF + jj;
-          const ChV dv = lds_ch<float>(smd + St::D, jj, w.k);
-          const ChV xv = lds_ch<IO>(smk + St::X, jj, w.k);
-          const ChV gv = lds_ch<IO>(smk + St::G, jj, w.k);
-          const float* brow = bck + St::BC / 4 + jj * NBC;
-          const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
-          const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
-          const ulonglong2 c01 = *reinterpret_cast<const ulonglong2*>(brow + NS);
-          const ulonglong2 c23 = *reinterpret_cast<const ulonglong2*>(brow + NS + 4);
-          const u64 Bp[4] = {b01.x, b01.y, b23.x, b23.y};
-          const u64 Cp[4] = {c01.x, c01.y, c23.x, c23.y};
-          float dd[NCH], xs[NCH];
-          u64 d2[NCH], dx2[NCH], g2[NCH];
+        for (int u = 0; u < NU; ++u) mu[u] = fma2(g2[u / 4], Cp[u % 4], mu[u]);
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) dsumc[c] += dd[c];
+        if (WIN && chunk_live) {
+          // exact exit of token t2 = t + Tbar from the window: subtract W_i gC_{t2},
+          // W_i = exp(A * sum_{j=i+1..t2} Delta_j); masked out when t2 >= T
+          const float wm = j < nwin ? 1.f : 0.f;
+          const ChV d2v = lds_ch<float>(sm + St::D2, j, w.k);
+          const ChV g2v = lds_ch<IO>(sm + St::G2, j, w.k);
+          const float* crow = reinterpret_cast<const float*>(sm + St::BC2) + 8 * w.half + j * NBC + NS;
+          const ulonglong2 e01 = *reinterpret_cast<const ulonglong2*>(crow);
+          const ulonglong2 e23 = *reinterpret_cast<const ulonglong2*>(crow + 4);
+          // rows of tokens past the sequence end are not staged: their C values must not be touched
+          const u64 C2p[4] = {wm != 0.f ? e01.x : 0ull, wm != 0.f ? e01.y : 0ull, wm != 0.f ? e23.x : 0ull,
+                              wm != 0.f ? e23.y : 0ull};
+          u64 ng2[NCH], sw2[NCH];
 #pragma unroll
           for (int c = 0; c < NCH; ++c) {
-            dd[c] = dv.v[c]; xs[c] = xv.v[c];
-            const float dxc = dv.v[c] * xv.v[c];
-            d2[c] = pk(dd[c], dd[c]); dx2[c] = pk(dxc, dxc); g2[c] = pk(gv.v[c], gv.v[c]);
+            const float swf = swc[c] + swl[c];
+            ng2[c] = pk(-g2v.v[c] * wm, -g2v.v[c] * wm);
+            sw2[c] = pk(swf, swf);
+            swl[c] += dd[c] - d2v.v[c] * wm;   // window of token t-1: (t-1, t-1+Tbar]
           }
-          // mu_i += g_i C_i   (mu already carries abar_{i+1} mu_{i+1})
 #pragma unroll
-          for (int u = 0; u < NU; ++u) mu[u] = fma2(g2[u / 4], Cp[u % 4], mu[u]);
-#pragma unroll
-          for (int c = 0; c < NCH; ++c) dsumc[c] += dd[c];
-          if (WIN && chunk_live) {
-            // exact exit of token t2 = t + Tbar from the window: subtract W_i gC_{t2},
-            // W_i = exp(A * sum_{j=i+1..t2} Delta_j); masked out when t2 >= T
-            const float wm = j < nwin ? 1.f : 0.f;
-            const ChV d2v = lds_ch<float>(smd + St::D2, jj, w.k);
-            const ChV g2v = lds_ch<IO>(smk + St::G2, jj, w.k);
-            const float* crow = bck + St::BC2 / 4 + jj * NBC + NS;
-            const ulonglong2 e01 = *reinterpret_cast<const ulonglong2*>(crow);
-            const ulonglong2 e23 = *reinterpret_cast<const ulonglong2*>(crow + 4);
-            // rows of tokens past the sequence end are not staged: their C values must not be touched
-            const u64 C2p[4] = {wm != 0.f ? e01.x : 0ull, wm != 0.f ? e01.y : 0ull, wm != 0.f ? e23.x : 0ull,
-                                wm != 0.f ? e23.y : 0ull};
-            u64 ng2[NCH], sw2[NCH];
-#pragma unroll
-            for (int c = 0; c < NCH; ++c) {
-              const float swf = swc[c] + swl[c];
-              ng2[c] = pk(-g2v.v[c] * wm, -g2v.v[c] * wm);
-              sw2[c] = pk(swf, swf);
-              swl[c] += dd[c] - d2v.v[c] * wm;   // window of token t-1: (t-1, t-1+Tbar]
-            }
-#pragma unroll
-            for (int u = 0; u < NU; ++u)
-              mu[u] = fma2(ex2_2(mul2(sw2[u / 4], A2[u])), mul2(ng2[u / 4], C2p[u % 4]), mu[u]);
-          }
-          u64 vB[4], vC[4];
-          float ssum[NCH], dsum[NCH];
+          for (int u = 0; u < NU; ++u)
+            mu[u] = fma2(ex2_2(mul2(sw2[u / 4], A2[u])), mul2(ng2[u / 4], C2p[u % 4]), mu[u]);
+        }
+        u64 vB[4], vC[4];
+        float ssum[NCH], dsum[NCH];
+        auto units = [&](auto rebuild) {
 #pragma unroll
           for (int ch = 0; ch < NCH; ++ch) {
             u64 sacc = 0ull, dacc = 0ull;
@@ -824,9 +910,8 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
               const int u = ch * 4 + m;
               const u64 a = ex2_2(mul2(d2[ch], A2[u]));
               const u64 bx = mul2(dx2[ch], Bp[m]);
-              u64 hn, hb;                                        // h_i and abar_i h_{i-1}
-              if (jj & 1) { hb = mul2(a, cur[jj / 2][u]); hn = fma2(a, cur[jj / 2][u], bx); }
-              else { hn = cur[jj / 2][u]; hb = fma2(bx, pk(-1.f, -1.f), hn); }
+              const u64 hn = decltype(rebuild)::v ? fma2(a, h[u], bx) : hT[u];   // h_i
+              const u64 hb = fma2(bx, pk(-1.f, -1.f), hn);                       // abar_i h_{i-1}
               vB[m] = ch == 0 ? mul2(mu[u], dx2[ch]) : fma2(mu[u], dx2[ch], vB[m]);   // dB partial (two channels)
               vC[m] = ch == 0 ? mul2(g2[ch], hn) : fma2(g2[ch], hn, vC[m]);           // dC partial
               sacc = fma2(mu[u], Bp[m], sacc);
@@ -838,48 +923,49 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
             ssum[ch] = hsum(sacc);
             dsum[ch] = hsum(dacc);
           }
+        };
+        if (j == CK - 1) units(BoolC<true>{}); else units(BoolC<false>{});
 #pragma unroll
-          for (int ch = 0; ch < NCH; ++ch) {
-            ssum[ch] += __shfl_xor_sync(0xffffffffu, ssum[ch], 1);
-            dsum[ch] += __shfl_xor_sync(0xffffffffu, dsum[ch], 1);
+        for (int ch = 0; ch < NCH; ++ch) {
+          ssum[ch] += __shfl_xor_sync(0xffffffffu, ssum[ch], 1);
+          dsum[ch] += __shfl_xor_sync(0xffffffffu, dsum[ch], 1);
+        }
+        {
+          const float d = dd[chf], xx = xs[chf];
+          const float sv = ssum[chf], dsv = dsum[chf];
+          const float ddelta = fmaf(dsv, LN2, xx * sv);
+          const float duv = ddelta * sig_from_delta(d);
+          dbacc += duv;
+          if (fin && j < nt) {
+            st_io<IO>(du_p, duv);
+            st_io<IO>(dx_p, d * sv);
           }
-          {
-            const float d = dd[chf], xx = xs[chf];
-            const float sv = ssum[chf], dsv = dsum[chf];
-            const float ddelta = fmaf(dsv, LN2, xx * sv);
-            const float duv = ddelta * sig_from_delta(d);
-            dbacc += duv;
-            if (fin && j < nt) {
-              st_io<IO>(du_p, duv);
-              st_io<IO>(dx_p, d * sv);
-            }
-            du_p -= du_ld;
-            dx_p -= P;
+          du_p -= du_ld;
+          dx_p -= P;
+        }
+        // sum over the warp's 16 channel pairs: every lane parks its 16 partials (dB[8*half+0..7], dC[8*half+0..7])
+        // in shared memory, then lane l adds up value (l >> 1) over the 16 lanes of its parity.  Quarter-blocks
+        // of 4 values are 544 bytes apart so that both the 16-byte stores and the 4-byte loads are conflict-free.
+        {
+          float* wr = wred[warp];
+          __syncwarp();   // the previous token's loads from wr are done
+#pragma unroll
+          for (int m = 0; m < 4; ++m) {
+            *reinterpret_cast<u64*>(wr + (m >> 1) * WRED_Q + lane * 4 + 2 * (m & 1)) = vB[m];
+            *reinterpret_cast<u64*>(wr + (2 + (m >> 1)) * WRED_Q + lane * 4 + 2 * (m & 1)) = vC[m];
           }
-          // sum over the warp's 16 channel pairs: every lane parks its 16 partials (dB[8*half+0..7], dC[8*half+0..7])
-          // in shared memory, then lane l adds up value (l >> 1) over the 16 lanes of its parity.  Quarter-blocks
-          // of 4 values are 544 bytes apart so that both the 16-byte stores and the 4-byte loads are conflict-free.
-          {
-            float* wr = wred[warp];
-            __syncwarp();   // the previous token's loads from wr are done
+          __syncwarp();
+          const int vi = lane >> 1;
+          const float* rd = wr + (vi >> 2) * WRED_Q + (lane & 1) * 4 + (vi & 3);
+          float part[16];
 #pragma unroll
-            for (int m = 0; m < 4; ++m) {
-              *reinterpret_cast<u64*>(wr + (m >> 1) * WRED_Q + lane * 4 + 2 * (m & 1)) = vB[m];
-              *reinterpret_cast<u64*>(wr + (2 + (m >> 1)) * WRED_Q + lane * 4 + 2 * (m & 1)) = vC[m];
-            }
-            __syncwarp();
-            const int vi = lane >> 1;
-            const float* rd = wr + (vi >> 2) * WRED_Q + (lane & 1) * 4 + (vi & 3);
-            float part[16];
+          for (int i2 = 0; i2 < 16; ++i2) part[i2] = rd[i2 * 8];
 #pragma unroll
-            for (int i2 = 0; i2 < 16; ++i2) part[i2] = rd[i2 * 8];
+          for (int wdt = 8; wdt >= 1; wdt >>= 1)   // pairwise tree: 4 dependent adds instead of 16
 #pragma unroll
-            for (int wdt = 8; wdt >= 1; wdt >>= 1)   // pairwise tree: 4 dependent adds instead of 16
-#pragma unroll
-              for (int i2 = 0; i2 < wdt; ++i2) part[i2] += part[i2 + wdt];
-            const float tot = part[0];
-            atomicAdd(&red[rb][j][(vi & 8) * 2 + 8 * w.half + (vi & 7)], tot);
-          }
+            for (int i2 = 0; i2 < wdt; ++i2) part[i2] += part[i2 + wdt];
+          const float tot = part[0];
+          atomicAdd(&red[rb][j][(vi & 8) * 2 + 8 * w.half + (vi & 7)], tot);
         }
       }
     }
@@ -888,11 +974,8 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
       for (int c = 0; c < NCH; ++c) sw[c] += (double)(dsumc[c] - sd2[c]);   // window sum at the previous chunk's last token
     }
     (void)swl;
-    const int bad = __syncthreads_or(ok ? 0 : 1);
-    if (bad) {
-      if (w.tid == 0) atomicExch(status, AS_ERR_TIMEOUT);
-      return;
-    }
+    const int bad = __syncthreads_or((ok && !tfail) ? 0 : 1);
+    if (bad) { failed = true; break; }
     if (w.tid == 0 && i + NSTAGE_MAIN < nchunk) issue(i + NSTAGE_MAIN);
     for (int e = w.tid; e < CK * NBC; e += NTHR) {
       const int j = e / NBC, q = e % NBC;
@@ -901,18 +984,28 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
       if (j < nt) atomicAdd(dbc + ((int64_t)b * T + tc + j) * NBC + q, sum);
     }
   }
-  if (w.act) {
+  if (failed) {
+    if (w.tid == 0) atomicExch(status, AS_ERR_TIMEOUT);
+  } else {
+    if (w.act) {
 #pragma unroll
-    for (int u = 0; u < NU; ++u) {
-      float alo, ahi, vlo, vhi;
-      upk(A2[u], alo, ahi);
-      upk(dAacc[u], vlo, vhi);
-      float* dst = dA_log + (int64_t)(w.pa + u / 4) * NS + 8 * w.half + 2 * (u % 4);
-      atomicAdd(dst, vlo * (alo * LN2));
-      atomicAdd(dst + 1, vhi * (ahi * LN2));
+      for (int u = 0; u < NU; ++u) {
+        float alo, ahi, vlo, vhi;
+        upk(A2[u], alo, ahi);
+        upk(dAacc[u], vlo, vhi);
+        float* dst = dA_log + (int64_t)(w.pa + u / 4) * NS + 8 * w.half + 2 * (u % 4);
+        atomicAdd(dst, vlo * (alo * LN2));
+        atomicAdd(dst + 1, vhi * (ahi * LN2));
+      }
     }
+    if (fin) atomicAdd(db_delta + pmine, dbacc);
   }
-  if (fin) atomicAdd(db_delta + pmine, dbacc);
+  // give the tensor memory back (every exit path comes through here)
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base_s), "n"(TM_COLS) : "memory");
+  }
 }
 
 // Self test of the bounded wait: one warp waits for a phase of an mbarrier that nothing will ever complete, with a
@@ -996,8 +1089,7 @@ template <typename IO, bool FULL>
 int launch_main_t(const Plan& pl, const ScanPtrs& sp, float* dA_log, float* db_delta, cudaStream_t st) {
   Maps m;
   if (make_maps(pl, sp, &m)) return 1;
-  using St = Stage<sizeof(IO), true, true, !FULL>;
-  const int bytes = NSTAGE_MAIN * St::BYTES + 128;
+  const int bytes = MainCfg<sizeof(IO), !FULL>::SMEM_DYN;
   auto kern = adjoint_main_kernel<IO, FULL>;
   static bool once = false;
   if (!once) { if (set_smem(kern, bytes)) return 1; once = true; }
