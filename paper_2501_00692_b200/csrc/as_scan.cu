@@ -190,6 +190,20 @@ template <> __device__ __forceinline__ ChV lds_ch<__nv_bfloat16>(const uint8_t* 
   }
   return r;
 }
+// the same from a pointer that already addresses this thread's channels in the row
+template <typename IO> __device__ __forceinline__ ChV lds_chp(const uint8_t* p);
+template <> __device__ __forceinline__ ChV lds_chp<float>(const uint8_t* p) {
+  ChV r;
+  const float2 t = *reinterpret_cast<const float2*>(p);
+  r.v[0] = t.x; r.v[NCH - 1] = t.y;
+  return r;
+}
+template <> __device__ __forceinline__ ChV lds_chp<__nv_bfloat16>(const uint8_t* p) {
+  ChV r;
+  const float2 t = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(p));
+  r.v[0] = t.x; r.v[NCH - 1] = t.y;
+  return r;
+}
 // NCH consecutive floats of a global per-channel array
 __device__ __forceinline__ ChV ldg_ch(const float* p) {
   ChV r;
@@ -399,7 +413,7 @@ __global__ void __launch_bounds__(NTHR) ascend_kernel(const __grid_constant__ CU
           // the two lanes of a pair hold the same sums: lane `half` writes channel `half` (one channel per thread: lane 0)
           const int chf = NCH == 2 ? w.half : 0;
           if (w.act && j < nt && (NCH == 2 || w.half == 0))
-            st_io<IO>(y + ((int64_t)b * pl.T + tc + j) * P + w.pa + chf, yv[chf]);
+            st_io<IO>(y + ((int64_t)b * pl.T + tc + j) * P + w.pa + chf, chf ? yv[NCH - 1] : yv[0]);
         }
         if (MU && j == jr) {
 #pragma unroll
@@ -845,21 +859,24 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
       // output rows of this chunk, walked from its last token down
       IO* du_p = du + ((int64_t)b * T + tc + (CK - 1)) * du_ld;
       IO* dx_p = dxdir + ((int64_t)b * T + tc + (CK - 1)) * P;
-      const float* bck = reinterpret_cast<const float*>(sm + St::BC) + 8 * w.half;
       // backward walk.  Token 7's state is rebuilt from the state after token 6 (still in h); the others come back
-      // from tensor memory.  abar_i h_{i-1} is formed as h_i - Delta_i x_i B_i.
+      // from tensor memory.  abar_i h_{i-1} is formed as h_i - Delta_i x_i B_i.  Row pointers walk down with the token.
+      const uint8_t* pD = sm + St::D + (CK - 1) * CH * 4 + 4 * NCH * w.k;       // Delta row (fp32)
+      const uint8_t* pX = sm + St::X + (CK - 1) * CH * ESZ + ESZ * NCH * w.k;   // x row; dy row at + (St::G - St::X)
+      const float* pB = reinterpret_cast<const float*>(sm + St::BC) + 8 * w.half + (CK - 1) * NBC;   // [B | C] row
+      float* pR = &red[rb][CK - 1][((lane >> 1) & 8) * 2 + 8 * w.half + ((lane >> 1) & 7)];
+      uint32_t tmj = tm + 16 * (CK - 2);
 #pragma unroll HALF
       for (int j = CK - 1; j >= 0; --j) {
         u64 hT[NU];
-        if (j < CK - 1) tmem_ld16(tm + 16 * j, hT);
-        const ChV dv = lds_ch<float>(sm + St::D, j, w.k);
-        const ChV xv = lds_ch<IO>(sm + St::X, j, w.k);
-        const ChV gv = lds_ch<IO>(sm + St::G, j, w.k);
-        const float* brow = bck + j * NBC;
-        const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(brow);
-        const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(brow + 4);
-        const ulonglong2 c01 = *reinterpret_cast<const ulonglong2*>(brow + NS);
-        const ulonglong2 c23 = *reinterpret_cast<const ulonglong2*>(brow + NS + 4);
+        if (j < CK - 1) { tmem_ld16(tmj, hT); tmj -= 16; }
+        const ChV dv = lds_chp<float>(pD);
+        const ChV xv = lds_chp<IO>(pX);
+        const ChV gv = lds_chp<IO>(pX + (St::G - St::X));
+        const ulonglong2 b01 = *reinterpret_cast<const ulonglong2*>(pB);
+        const ulonglong2 b23 = *reinterpret_cast<const ulonglong2*>(pB + 4);
+        const ulonglong2 c01 = *reinterpret_cast<const ulonglong2*>(pB + NS);
+        const ulonglong2 c23 = *reinterpret_cast<const ulonglong2*>(pB + NS + 4);
         const u64 Bp[4] = {b01.x, b01.y, b23.x, b23.y};
         const u64 Cp[4] = {c01.x, c01.y, c23.x, c23.y};
         float dd[NCH], xs[NCH];
@@ -879,9 +896,9 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
           // exact exit of token t2 = t + Tbar from the window: subtract W_i gC_{t2},
           // W_i = exp(A * sum_{j=i+1..t2} Delta_j); masked out when t2 >= T
           const float wm = j < nwin ? 1.f : 0.f;
-          const ChV d2v = lds_ch<float>(sm + St::D2, j, w.k);
-          const ChV g2v = lds_ch<IO>(sm + St::G2, j, w.k);
-          const float* crow = reinterpret_cast<const float*>(sm + St::BC2) + 8 * w.half + j * NBC + NS;
+          const ChV d2v = lds_chp<float>(pD + (St::D2 - St::D));
+          const ChV g2v = lds_chp<IO>(pX + (St::G2 - St::X));
+          const float* crow = pB + (St::BC2 - St::BC) / 4 + NS;
           const ulonglong2 e01 = *reinterpret_cast<const ulonglong2*>(crow);
           const ulonglong2 e23 = *reinterpret_cast<const ulonglong2*>(crow + 4);
           // rows of tokens past the sequence end are not staged: their C values must not be touched
@@ -931,8 +948,8 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
           dsum[ch] += __shfl_xor_sync(0xffffffffu, dsum[ch], 1);
         }
         {
-          const float d = dd[chf], xx = xs[chf];
-          const float sv = ssum[chf], dsv = dsum[chf];
+          const float d = chf ? dd[NCH - 1] : dd[0], xx = chf ? xs[NCH - 1] : xs[0];   // selects, not indexed local arrays
+          const float sv = chf ? ssum[NCH - 1] : ssum[0], dsv = chf ? dsum[NCH - 1] : dsum[0];
           const float ddelta = fmaf(dsv, LN2, xx * sv);
           const float duv = ddelta * sig_from_delta(d);
           dbacc += duv;
@@ -965,8 +982,9 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
 #pragma unroll
             for (int i2 = 0; i2 < wdt; ++i2) part[i2] += part[i2 + wdt];
           const float tot = part[0];
-          atomicAdd(&red[rb][j][(vi & 8) * 2 + 8 * w.half + (vi & 7)], tot);
+          atomicAdd(pR, tot);
         }
+        pD -= CH * 4; pX -= CH * ESZ; pB -= NBC; pR -= NBC;
       }
     }
     if (WIN) {
