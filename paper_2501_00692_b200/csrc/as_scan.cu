@@ -880,12 +880,12 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         const u64 Bp[4] = {b01.x, b01.y, b23.x, b23.y};
         const u64 Cp[4] = {c01.x, c01.y, c23.x, c23.y};
         float dd[NCH], xs[NCH];
-        u64 d2[NCH], dx2[NCH], g2[NCH];
+        u64 d2[NCH], dx2[NCH], ndx2[NCH], g2[NCH];
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
           dd[c] = dv.v[c]; xs[c] = xv.v[c];
           const float dxc = dv.v[c] * xv.v[c];
-          d2[c] = pk(dd[c], dd[c]); dx2[c] = pk(dxc, dxc); g2[c] = pk(gv.v[c], gv.v[c]);
+          d2[c] = pk(dd[c], dd[c]); dx2[c] = pk(dxc, dxc); ndx2[c] = pk(-dxc, -dxc); g2[c] = pk(gv.v[c], gv.v[c]);
         }
         // mu_i += g_i C_i   (mu already carries abar_{i+1} mu_{i+1})
 #pragma unroll
@@ -921,19 +921,19 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         auto units = [&](auto rebuild) {
 #pragma unroll
           for (int ch = 0; ch < NCH; ++ch) {
-            u64 sacc = 0ull, dacc = 0ull;
+            u64 sacc, dacc;
 #pragma unroll
             for (int m = 0; m < 4; ++m) {
               const int u = ch * 4 + m;
               const u64 a = ex2_2(mul2(d2[ch], A2[u]));
-              const u64 bx = mul2(dx2[ch], Bp[m]);
-              const u64 hn = decltype(rebuild)::v ? fma2(a, h[u], bx) : hT[u];   // h_i
-              const u64 hb = fma2(bx, pk(-1.f, -1.f), hn);                       // abar_i h_{i-1}
+              u64 hn, hb;   // h_i and abar_i h_{i-1} = h_i - Delta_i x_i B_i
+              if (decltype(rebuild)::v) { hb = mul2(a, h[u]); hn = fma2(dx2[ch], Bp[m], hb); }
+              else { hn = hT[u]; hb = fma2(ndx2[ch], Bp[m], hn); }
               vB[m] = ch == 0 ? mul2(mu[u], dx2[ch]) : fma2(mu[u], dx2[ch], vB[m]);   // dB partial (two channels)
               vC[m] = ch == 0 ? mul2(g2[ch], hn) : fma2(g2[ch], hn, vC[m]);           // dC partial
-              sacc = fma2(mu[u], Bp[m], sacc);
+              sacc = m == 0 ? mul2(mu[u], Bp[m]) : fma2(mu[u], Bp[m], sacc);
               const u64 q = mul2(mu[u], hb);
-              dacc = fma2(q, A2[u], dacc);
+              dacc = m == 0 ? mul2(q, A2[u]) : fma2(q, A2[u], dacc);
               dAacc[u] = fma2(q, d2[ch], dAacc[u]);
               mu[u] = mul2(mu[u], a);                                                  // ready for token i-1
             }

@@ -14,18 +14,21 @@ def theta_f64(theta):
     return {k: synth.to_f64(v) for k, v in theta.items()}
 
 
-def errors(got, want):
-    """(relative L2 error, max-abs error relative to max-abs of the oracle)."""
+def errors(got, want, floor=0.0):
+    """(relative L2 error, max-abs error relative to max-abs of the oracle).
+
+    `floor` is a lower bound on the reference magnitude used in both ratios (per element for the max, times
+    sqrt(size) for the L2 norm): it is only needed where the reference is identically zero because terms cancel."""
     got = np.asarray(got, dtype=np.float64); want = np.asarray(want, dtype=np.float64)
     d = got - want
-    l2 = np.linalg.norm(d.ravel()) / max(np.linalg.norm(want.ravel()), 1e-300)
-    mx = np.abs(d).max() / max(np.abs(want).max(), 1e-300)
+    l2 = np.linalg.norm(d.ravel()) / max(np.linalg.norm(want.ravel()), floor * np.sqrt(max(want.size, 1)), 1e-300)
+    mx = np.abs(d).max() / max(np.abs(want).max(), floor, 1e-300)
     return l2, mx
 
 
-def assert_close(got, want, tol, what=""):
+def assert_close(got, want, tol, what="", floor=0.0):
     assert np.isfinite(np.asarray(got, dtype=np.float64)).all(), f"{what}: non-finite values"
-    l2, mx = errors(got, want)
+    l2, mx = errors(got, want, floor)
     assert l2 <= tol and mx <= tol, f"{what}: rel-L2 {l2:.3e}, rel-max {mx:.3e} > {tol}"
     return l2, mx
 
@@ -61,10 +64,13 @@ def oracle_adjoint(theta, x, dy, tbar, tier="block", channel_block=None):
                      channel_block=channel_block)
 
 
-def compare_grads(g, ref, tol, keys=PARAM + ("dx",)):
+def compare_grads(g, ref, tol, keys=PARAM + ("dx",), zero_floor=None):
+    """`zero_floor` maps a gradient name to the magnitude its error is measured against when the oracle's value
+    is identically zero (see `errors`)."""
     res = {}
     for k in keys:
         if g.get(k) is None:
             continue
-        res[k] = assert_close(synth.to_f64(g[k]), ref[k], tol, k)
+        fl = (zero_floor or {}).get(k, 0.0) if not np.any(ref[k]) else 0.0
+        res[k] = assert_close(synth.to_f64(g[k]), ref[k], tol, k, floor=fl)
     return res

@@ -136,7 +136,11 @@ def test_degenerate_and_tiny_shapes(batch, T, P, tbar, io):
     w = synth.custom_workload("tiny", 16, batch, T, P, tbar=tbar, io=io)
     theta, x, dy = setup(w, slow=True)
     ref = oracle_adjoint(theta, x, dy, tbar, tier="direct")
-    compare_grads(gpu_adjoint(w, theta, x, dy, tbar), ref, TOL[io])
+    # With a single token dA_log is identically zero (h_0 = 0).  The library forms abar_t h_{t-1} as
+    # h_t - Delta_t x_t B_t with one rounding, so its error is relative to |h_t|, not to the vanishing difference:
+    # measure it against the size of the other state-dependent gradient, dW_B.
+    zf = {"dA_log": float(np.abs(ref["dW_B"]).max())}
+    compare_grads(gpu_adjoint(w, theta, x, dy, tbar), ref, TOL[io], zero_floor=zf)
     y = gpu_forward(w, theta, x)
     assert_close(synth.to_f64(y), ref["y"], TOL[io], "y")
     gb = gpu_adjoint(w, theta, x, dy, T, bptt=True)
