@@ -368,9 +368,7 @@ __global__ void __launch_bounds__(NTHR) ascend_kernel(const __grid_constant__ CU
       }
       __syncthreads();
     }
-    if (ok) {
-#pragma unroll
-      for (int j = 0; j < CK; ++j) {
+    auto token = [&](int j) {
         // channels past P read the zero fill of the TMA box: Delta = x = g = 0 keeps their slots at zero
         const ChV dv = lds_ch<float>(sm + St::D, j, w.k);
         const ChV xv = lds_ch<IO>(sm + St::X, j, w.k);
@@ -415,12 +413,23 @@ __global__ void __launch_bounds__(NTHR) ascend_kernel(const __grid_constant__ CU
           if (w.act && j < nt && (NCH == 2 || w.half == 0))
             st_io<IO>(y + ((int64_t)b * pl.T + tc + j) * P + w.pa + chf, chf ? yv[NCH - 1] : yv[0]);
         }
-        if (MU && j == jr) {
+    };
+    if (ok) {
+      if (MU && jr >= 0 && jr < CK) {
+        // the one chunk of the segment that holds its r-th token: take the snapshot right after that token
+#pragma unroll 1
+        for (int j = 0; j < CK; ++j) {
+          token(j);
+          if (j == jr) {
 #pragma unroll
-          for (int c = 0; c < NCH; ++c) partd[c] = cum[c];
+            for (int c = 0; c < NCH; ++c) partd[c] = cum[c];
 #pragma unroll
-          for (int u = 0; u < NU; ++u) snap[u] = acc[u];
+            for (int u = 0; u < NU; ++u) snap[u] = acc[u];
+          }
         }
+      } else {
+#pragma unroll
+        for (int j = 0; j < CK; ++j) token(j);
       }
     }
     const int bad = __syncthreads_or(ok ? 0 : 1);
