@@ -161,7 +161,7 @@ struct Stage {
 constexpr int NSTAGE = 3;        // ascending kernels
 constexpr int WRED_Q = 32 * 4 + 8;   // floats per quarter-block of the per-warp reduction scratch (512 B + 32 B skew)
 constexpr int MAIN_CTAS = 3;    // resident CTAs per SM the main kernel is compiled for (168 registers per thread)
-constexpr int HALF = CK / 2;       // unroll factor of the main adjoint kernel's backward token loop
+constexpr int BW_UNROLL = 4;     // unroll factor of the main adjoint kernel's backward token loop
 constexpr int NSTAGE_MAIN = 2;   // main adjoint kernel: a chunk takes thousands of cycles, one chunk of lookahead suffices
 
 // per-thread values of its NCH channels
@@ -568,22 +568,12 @@ __global__ void __launch_bounds__(NTHR) fixup_mu_kernel(Plan pl, const float* __
   }
 }
 
-// ------------------------------------------------------------------------------------------------
-// main adjoint kernel: descending over the CK-token chunks of one segment.
-//   per chunk: rebuild h for the chunk from its checkpoint (keeping only every other token's state in
-//   registers; the odd tokens' states are rebuilt in the backward walk from the abar they need anyway),
-//   then walk it backwards updating the summed cotangent
-//       mu_i = gC_i + abar_{i+1} mu_{i+1} - W_i gC_{i+Tbar}
-//   and evaluating the per-token VJPs.
-// ------------------------------------------------------------------------------------------------
-template <bool B> struct BoolC { static constexpr bool v = B; };
 // ---- tensor memory as a per-thread scratchpad ------------------------------------------------------
 // The main adjoint kernel runs no MMA, so the SM's tensor memory is free.  Each CTA allocates 128 of the 512
-// columns of its SM (three CTAs are resident) and every thread parks per-token states in its own TMEM lane:
+// columns of its SM (three CTAs are resident) and every thread parks the chunk's eight states in its own TMEM lane:
 // warp w of the 4-warp CTA owns lanes [32w, 32w+32), a 32x32b access moves 16 registers of each lane to or
 // from 16 consecutive columns.
-constexpr int TM_COLS = 128;
-constexpr int TM_HST = 7 * 16;   // columns [16 j, 16 j + 16): state after token j (j = 0..6); [112, 128): segment-start state
+constexpr int TM_COLS = CK * 16;   // columns [16 j, 16 j + 16): state after token j of the current chunk
 
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const u64 (&v)[NU]) {
   uint32_t r[16];
@@ -648,7 +638,7 @@ template <int ESZ, bool WIN> struct MainCfg {
 
 // ------------------------------------------------------------------------------------------------
 // main adjoint kernel: one CTA per (channel tile, segment, batch element), chunks walked last to first.
-// Per chunk: rebuild the states after tokens 0..6 from the chunk checkpoint and park them in tensor memory,
+// Per chunk: rebuild the states after its eight tokens from the chunk checkpoint and park them in tensor memory,
 // then walk the chunk's tokens backwards: mu recurrence (with the exact window exit), the per-token
 // vector-Jacobian products, the channel sums dB_t / dC_t, and the per-channel outputs du_t and dx_dir_t.
 // ------------------------------------------------------------------------------------------------
@@ -668,6 +658,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   __shared__ uint32_t tmem_base_s;
   __shared__ float red[2][CK][NBC];                 // per-token [dB | dC] sums of the CTA, two chunks in flight
   __shared__ __align__(16) float wred[NTHR / 32][4 * WRED_Q];   // per-warp scratch of the channel reduction
+  __shared__ ulonglong2 hst_s[2 * NCH][NTHR];       // true segment-start state, read back once per chunk
   uint8_t* smem = smem_raw + ((128u - (smem_u32(smem_raw) & 127u)) & 127u);   // stays a shared-space pointer
   uint8_t* ckp_s = smem + NSTAGE_MAIN * St::BYTES;
 
@@ -755,11 +746,11 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   load_A2(A_log, w, A2);
   const int64_t sb = ((int64_t)b * pl.S + s) * pl.tiles + tile;
   load_block_g(reinterpret_cast<const float*>(ws + pl.off_carry) + sb * TILE_FLOATS, w.tid, mu);
-  {   // true segment-start state: parked in tensor memory, read back once per chunk
+  {   // true segment-start state: parked in shared memory
     u64 hst[NU];
     load_block_g(reinterpret_cast<const float*>(ws + pl.off_hstart) + sb * TILE_FLOATS, w.tid, hst);
-    tmem_st16(tm + TM_HST, hst);
-    tmem_wait_st();
+#pragma unroll
+    for (int q = 0; q < 2 * NCH; ++q) hst_s[q][w.tid] = make_ulonglong2(hst[2 * q], hst[2 * q + 1]);
   }
 #pragma unroll
   for (int u = 0; u < NU; ++u) dAacc[u] = 0ull;
@@ -815,7 +806,11 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
       mbar_arrive(&ckp_free);   // this thread is done with the checkpoint buffer
       {
         u64 hst[NU], c2[NCH];
-        tmem_ld16(tm + TM_HST, hst);
+#pragma unroll
+        for (int q = 0; q < 2 * NCH; ++q) {
+          const ulonglong2 hq = hst_s[q][w.tid];
+          hst[2 * q] = hq.x; hst[2 * q + 1] = hq.y;
+        }
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
           float csv = *reinterpret_cast<const float*>(sm + St::CS + 4 * (NCH * w.k + c));
@@ -841,11 +836,11 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         for (int c = 0; c < NCH; ++c) live = live || ((swc[c] - sd2[c]) * a2max[c] > -64.f);
         chunk_live = __any_sync(0xffffffffu, live && w.act && nwin > 0);
       }
-      // forward rebuild: the states after tokens 0..6 go to tensor memory; the one after token 6 also stays in h
+      // forward rebuild: the states after the chunk's eight tokens go to tensor memory
       {
         const float* bck = reinterpret_cast<const float*>(sm + St::BC) + 8 * w.half;
 #pragma unroll 1
-        for (int j = 0; j < CK - 1; ++j) {
+        for (int j = 0; j < CK; ++j) {
           const ChV dv = lds_ch<float>(sm + St::D, j, w.k);
           const ChV xv = lds_ch<IO>(sm + St::X, j, w.k);
           const float* brow = bck + j * NBC;
@@ -872,17 +867,18 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
       // output rows of this chunk, walked from its last token down
       IO* du_p = fin ? du + ((int64_t)b * T + tc + (CK - 1)) * du_ld : dummy;
       IO* dx_p = fin ? dxdir + ((int64_t)b * T + tc + (CK - 1)) * P : dummy;
-      // backward walk.  Token 7's state is rebuilt from the state after token 6 (still in h); the others come back
-      // from tensor memory.  abar_i h_{i-1} is formed as h_i - Delta_i x_i B_i.  Row pointers walk down with the token.
+      // backward walk: h_i comes back from tensor memory, abar_i h_{i-1} is formed as h_i - Delta_i x_i B_i.
+      // Row pointers walk down with the token.
       const uint8_t* pD = sm + St::D + (CK - 1) * CH * 4 + 4 * NCH * w.k;       // Delta row (fp32)
       const uint8_t* pX = sm + St::X + (CK - 1) * CH * ESZ + ESZ * NCH * w.k;   // x row; dy row at + (St::G - St::X)
       const float* pB = reinterpret_cast<const float*>(sm + St::BC) + 8 * w.half + (CK - 1) * NBC;   // [B | C] row
       float* pR = &red[rb][CK - 1][((lane >> 1) & 8) * 2 + 8 * w.half + ((lane >> 1) & 7)];
-      uint32_t tmj = tm + 16 * (CK - 2);
-#pragma unroll HALF
+      uint32_t tmj = tm + 16 * (CK - 1);
+#pragma unroll BW_UNROLL
       for (int j = CK - 1; j >= 0; --j) {
         u64 hT[NU];
-        if (j < CK - 1) { tmem_ld16(tmj, hT); tmj -= 16; }
+        tmem_ld16(tmj, hT);
+        tmj -= 16;
         const ChV dv = lds_chp<float>(pD);
         const ChV xv = lds_chp<IO>(pX);
         const ChV gv = lds_chp<IO>(pX + (St::G - St::X));
@@ -931,30 +927,26 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         }
         u64 vB[4], vC[4];
         float ssum[NCH], dsum[NCH];
-        auto units = [&](auto rebuild) {
 #pragma unroll
-          for (int ch = 0; ch < NCH; ++ch) {
-            u64 sacc, dacc;
+        for (int ch = 0; ch < NCH; ++ch) {
+          u64 sacc, dacc;
 #pragma unroll
-            for (int m = 0; m < 4; ++m) {
-              const int u = ch * 4 + m;
-              const u64 a = ex2_2(mul2(d2[ch], A2[u]));
-              u64 hn, hb;   // h_i and abar_i h_{i-1} = h_i - Delta_i x_i B_i
-              if (decltype(rebuild)::v) { hb = mul2(a, h[u]); hn = fma2(dx2[ch], Bp[m], hb); }
-              else { hn = hT[u]; hb = fma2(ndx2[ch], Bp[m], hn); }
-              vB[m] = ch == 0 ? mul2(mu[u], dx2[ch]) : fma2(mu[u], dx2[ch], vB[m]);   // dB partial (two channels)
-              vC[m] = ch == 0 ? mul2(g2[ch], hn) : fma2(g2[ch], hn, vC[m]);           // dC partial
-              sacc = m == 0 ? mul2(mu[u], Bp[m]) : fma2(mu[u], Bp[m], sacc);
-              const u64 q = mul2(mu[u], hb);
-              dacc = m == 0 ? mul2(q, A2[u]) : fma2(q, A2[u], dacc);
-              dAacc[u] = fma2(q, d2[ch], dAacc[u]);
-              mu[u] = mul2(mu[u], a);                                                  // ready for token i-1
-            }
-            ssum[ch] = hsum(sacc);
-            dsum[ch] = hsum(dacc);
+          for (int m = 0; m < 4; ++m) {
+            const int u = ch * 4 + m;
+            const u64 a = ex2_2(mul2(d2[ch], A2[u]));
+            const u64 hn = hT[u];                                  // h_i
+            const u64 hb = fma2(ndx2[ch], Bp[m], hn);              // abar_i h_{i-1} = h_i - Delta_i x_i B_i
+            vB[m] = ch == 0 ? mul2(mu[u], dx2[ch]) : fma2(mu[u], dx2[ch], vB[m]);   // dB partial (two channels)
+            vC[m] = ch == 0 ? mul2(g2[ch], hn) : fma2(g2[ch], hn, vC[m]);           // dC partial
+            sacc = m == 0 ? mul2(mu[u], Bp[m]) : fma2(mu[u], Bp[m], sacc);
+            const u64 q = mul2(mu[u], hb);
+            dacc = m == 0 ? mul2(q, A2[u]) : fma2(q, A2[u], dacc);
+            dAacc[u] = fma2(q, d2[ch], dAacc[u]);
+            mu[u] = mul2(mu[u], a);                                                  // ready for token i-1
           }
-        };
-        if (j == CK - 1) units(BoolC<true>{}); else units(BoolC<false>{});
+          ssum[ch] = hsum(sacc);
+          dsum[ch] = hsum(dacc);
+        }
 #pragma unroll
         for (int ch = 0; ch < NCH; ++ch) {
           ssum[ch] += __shfl_xor_sync(0xffffffffu, ssum[ch], 1);
