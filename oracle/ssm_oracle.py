@@ -33,7 +33,8 @@ Pins (tests/test_oracle_pins.py): adjoint == hand BPTT; truncated == full for
 Tbar >= T; central finite differences; VJP counts incl. the printed 64 % figure;
 impulse window edges; windowed-BPTT brute force; Tbar = 1 closed form; LTI
 geometric closed forms; explicit O(T^2) forward sum; the C-VJP identity of
-Appendix A.3; linearity / permutation invariants; stack modes vs finite differences.
+Appendix A.3; linearity / permutation invariants; stack modes vs finite differences;
+scalar structure: masked T x T product form of the forward, finite differences of the tied rate.
 Unpinned by anything printed in the paper: absolute gradient values on the named
 workloads (the paper prints none), the RMSNorm epsilon, the error metric.
 """
@@ -285,6 +286,46 @@ def windowed_bptt_bruteforce(theta, x, g, tbar):
 
 # --------------------------------------------------------------------------- batches
 PARAM_GRADS = ("dW_delta", "db_delta", "dW_B", "dW_C", "dA_log")
+
+
+# ---------------------------------------------------------------------------------------------
+# scalar structure (the "Scalar SSM" row of Table 1, Section 4.5): one decay rate per channel,
+# A[p, n] = a[p] for every state n, so that A^t is a scalar multiple of the identity on each
+# channel's N states.  It is the diagonal layer with the N entries of a row of A_log tied together:
+# the forward is unchanged, and the gradient of a tied parameter is the sum of the gradients of
+# the entries it is tied to (chain rule).
+# ---------------------------------------------------------------------------------------------
+def untie_scalar_A(theta, N):
+    """theta with A_log [P] -> the equivalent diagonal theta with A_log [P,N] (rows constant)."""
+    th = dict(theta)
+    a = np.asarray(theta["A_log"], dtype=np.float64)
+    assert a.ndim == 1
+    th["A_log"] = np.repeat(a[:, None], N, axis=1)
+    return th
+
+
+def scalar_adjoint_grad(theta, x, g, tbar, N, **kw):
+    """Adjoint-method gradient of the scalar-structure layer for one sequence: dA_log is [P]."""
+    out = adjoint_grad(untie_scalar_A(theta, N), x, g, tbar, **kw)
+    out["dA_log"] = out["dA_log"].sum(axis=1)
+    return out
+
+
+def scalar_forward_quadratic(theta, x, N):
+    """Forward of the scalar-structure layer written as one masked T x T product per channel (no recurrence):
+        y_t[p] = sum_{j<=t} exp(a_p * sum_{i=j+1..t} Delta_i[p]) * (C_t . B_j) * Delta_j[p] x_j[p]
+    Used only to pin the recurrent forward; O(T^2 P)."""
+    a = -np.exp(np.asarray(theta["A_log"], dtype=np.float64))          # [P]
+    _, delta, Bm, Cm, _ = nets(untie_scalar_A(theta, N), x)
+    T, P = x.shape
+    G = Cm @ Bm.T                                                      # [T,T]  C_t . B_j
+    cum = np.cumsum(delta, axis=0)                                     # [T,P]
+    y = np.zeros((T, P))
+    for p in range(P):
+        L = np.exp(a[p] * (cum[:, None, p] - cum[None, :, p]))         # exp(a * sum_{i=j+1..t} Delta_i)
+        L = np.tril(L)
+        y[:, p] = (L * G) @ (delta[:, p] * x[:, p])
+    return y
 
 
 def batched(fn, theta, x, g, *args, **kw):

@@ -297,3 +297,47 @@ def test_stack_chained_equals_fd_and_paper_mode_is_detached():
         assert maxdiff(pg[k], ref, O.PARAM_GRADS) < 1e-12
     assert maxdiff(pg[K - 1], grads[K - 1], O.PARAM_GRADS) < 1e-12
     assert maxdiff(pg[0], grads[0], O.PARAM_GRADS) > 1e-4
+
+
+# ---- scalar structure (Table 1 "Scalar SSM": one decay rate per channel) -----------------------------------------
+def _scalar_theta(tiny):
+    th, x, g = tiny
+    ths = dict(th)
+    ths["A_log"] = th["A_log"][:, 0].copy()          # [P]
+    return ths, x, g, th["A_log"].shape[1]
+
+
+def test_scalar_forward_equals_masked_product_form(tiny):
+    # with A^t a multiple of the identity the recurrence collapses to y = (L o (C B^T)) (Delta x) per channel
+    ths, x, _, N = _scalar_theta(tiny)
+    y_rec = O.ssm_forward(O.untie_scalar_A(ths, N), x)
+    y_quad = O.scalar_forward_quadratic(ths, x, N)
+    assert np.abs(y_rec - y_quad).max() / np.abs(y_rec).max() < 1e-12
+
+
+def test_scalar_rate_gradient_by_finite_differences(tiny):
+    ths, x, g, N = _scalar_theta(tiny)
+    for tbar in (x.shape[0], 5):
+        a = O.scalar_adjoint_grad(ths, x, g, tbar, N)
+        assert a["dA_log"].shape == ths["A_log"].shape
+        if tbar < x.shape[0]:
+            continue          # the truncated form is not the gradient of a scalar loss: only its shape is checked here
+        eps = 1e-6
+        fd = np.zeros_like(ths["A_log"])
+        for p in range(fd.size):
+            tp = {k: v.copy() for k, v in ths.items()}; tm = {k: v.copy() for k, v in ths.items()}
+            tp["A_log"][p] += eps; tm["A_log"][p] -= eps
+            lp = float(np.sum(g * O.scalar_forward_quadratic(tp, x, N)))
+            lm = float(np.sum(g * O.scalar_forward_quadratic(tm, x, N)))
+            fd[p] = (lp - lm) / (2 * eps)
+        assert np.abs(fd - a["dA_log"]).max() / np.abs(a["dA_log"]).max() < 1e-7
+
+
+def test_scalar_truncated_rate_gradient_is_windowed_bptt(tiny):
+    # truncated form with tied rates against the brute-force per-token windowed backpropagation, tied the same way
+    ths, x, g, N = _scalar_theta(tiny)
+    a = O.scalar_adjoint_grad(ths, x, g, 5, N)
+    b = O.windowed_bptt_bruteforce(O.untie_scalar_A(ths, N), x, g, 5)
+    assert np.abs(a["dA_log"] - b["dA_log"].sum(axis=1)).max() / np.abs(a["dA_log"]).max() < 1e-10
+    for k in ("dW_delta", "dW_B", "dW_C", "db_delta", "dx"):
+        assert np.abs(a[k] - b[k]).max() / np.abs(b[k]).max() < 1e-10, k
