@@ -31,14 +31,19 @@
 extern "C" {
 #endif
 
-#define AS_VERSION 100
+#define AS_VERSION 101
 
 typedef enum { AS_F32 = 0, AS_BF16 = 1 } as_dtype_t;
+
+/* Structure of A (Table 1 of Section 4.5): AS_A_DIAGONAL, one decay rate per (channel, state), A_log [P,N];
+ * AS_A_SCALAR, one decay rate per channel shared by its N states ("Scalar SSM": A^t is a multiple of the identity on
+ * each channel), A_log [P] and dA_log [P] (the sum over n of the diagonal layer's dA_log[p,n]). */
+typedef enum { AS_A_DIAGONAL = 0, AS_A_SCALAR = 1 } as_structure_t;
 
 enum {
   AS_OK = 0,
   AS_ERR_NULL = -1,       /* a required pointer is NULL */
-  AS_ERR_SHAPE = -2,      /* non-positive dimension, or d_state != 16 */
+  AS_ERR_SHAPE = -2,      /* non-positive dimension, d_state != 16, or an unknown a_structure */
   AS_ERR_DTYPE = -3,      /* io is neither AS_F32 nor AS_BF16 */
   AS_ERR_TBAR = -4,       /* tbar < 1 */
   AS_ERR_WORKSPACE = -5,  /* ws_bytes smaller than as_workspace_bytes reports */
@@ -57,6 +62,7 @@ typedef struct {
   int32_t d_model;    /* P >= 8, multiple of 8 */
   int32_t d_state;    /* N, must be 16 */
   int32_t io;         /* as_dtype_t of x, y, dy, dx and the W_* matrices */
+  int32_t a_structure; /* as_structure_t */
 } as_shape_t;
 
 typedef struct {          /* parameters of one layer (device pointers) */
@@ -64,7 +70,7 @@ typedef struct {          /* parameters of one layer (device pointers) */
   const float *b_delta;   /* [P]   fp32 */
   const void  *W_B;       /* [N,P] io dtype */
   const void  *W_C;       /* [N,P] io dtype */
-  const float *A_log;     /* [P,N] fp32, A = -exp(A_log) */
+  const float *A_log;     /* [P,N] fp32 (AS_A_SCALAR: [P]), A = -exp(A_log) */
 } as_params_t;
 
 typedef struct {          /* gradient outputs (device pointers); parameter gradients are fp32, summed over the batch */
@@ -72,7 +78,7 @@ typedef struct {          /* gradient outputs (device pointers); parameter gradi
   float *db_delta;        /* [P]   */
   float *dW_B;            /* [N,P] */
   float *dW_C;            /* [N,P] */
-  float *dA_log;          /* [P,N] */
+  float *dA_log;          /* [P,N] (AS_A_SCALAR: [P]) */
   void  *dx;              /* [Bsz,T,P] io dtype, always overwritten; may be NULL (input gradient skipped) */
 } as_grads_t;
 

@@ -15,6 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libadjoint_ssm.so")
 
 AS_F32, AS_BF16 = 0, 1
+AS_A_DIAGONAL, AS_A_SCALAR = 0, 1
 AS_ACCUMULATE = 1
 AS_OK = 0
 AS_ERR_NULL, AS_ERR_SHAPE, AS_ERR_DTYPE, AS_ERR_TBAR = -1, -2, -3, -4
@@ -30,7 +31,7 @@ PHASES = ("projections", "prepass", "fixup", "adjoint_main", "weight_grads", "in
 
 class as_shape_t(C.Structure):
     _fields_ = [("batch", C.c_int32), ("seqlen", C.c_int64), ("d_model", C.c_int32),
-                ("d_state", C.c_int32), ("io", C.c_int32)]
+                ("d_state", C.c_int32), ("io", C.c_int32), ("a_structure", C.c_int32)]
 
 
 class as_params_t(C.Structure):
@@ -104,13 +105,13 @@ def _check(code: int, where: str):
         raise AsError(code, where)
 
 
-def make_shape(batch, seqlen, d_model, d_state=16, io=AS_F32) -> as_shape_t:
-    return as_shape_t(int(batch), int(seqlen), int(d_model), int(d_state), int(io))
+def make_shape(batch, seqlen, d_model, d_state=16, io=AS_F32, a_structure=AS_A_DIAGONAL) -> as_shape_t:
+    return as_shape_t(int(batch), int(seqlen), int(d_model), int(d_state), int(io), int(a_structure))
 
 
-def shape_of(x: torch.Tensor, d_state=16) -> as_shape_t:
+def shape_of(x: torch.Tensor, d_state=16, a_scalar=False) -> as_shape_t:
     io = {torch.float32: AS_F32, torch.bfloat16: AS_BF16}[x.dtype]
-    return make_shape(x.shape[0], x.shape[1], x.shape[2], d_state, io)
+    return make_shape(x.shape[0], x.shape[1], x.shape[2], d_state, io, AS_A_SCALAR if a_scalar else AS_A_DIAGONAL)
 
 
 def make_params(theta: dict) -> as_params_t:
@@ -122,7 +123,8 @@ def alloc_grads(shape: as_shape_t, device, with_dx=True) -> dict:
     P, N = shape.d_model, shape.d_state
     f = dict(dtype=torch.float32, device=device)
     g = {"dW_delta": torch.empty(P, P, **f), "db_delta": torch.empty(P, **f), "dW_B": torch.empty(N, P, **f),
-         "dW_C": torch.empty(N, P, **f), "dA_log": torch.empty(P, N, **f), "dx": None}
+         "dW_C": torch.empty(N, P, **f),
+         "dA_log": torch.empty(P, **f) if shape.a_structure == AS_A_SCALAR else torch.empty(P, N, **f), "dx": None}
     if with_dx:
         dt = torch.float32 if shape.io == AS_F32 else torch.bfloat16
         g["dx"] = torch.empty(shape.batch, shape.seqlen, P, dtype=dt, device=device)

@@ -25,6 +25,7 @@ int check_shape(const as_shape_t* sh) {
   if (!sh) return AS_ERR_NULL;
   if (sh->batch < 1 || sh->seqlen < 1 || sh->d_model < 1) return AS_ERR_SHAPE;
   if (sh->d_state != NS) return AS_ERR_SHAPE;
+  if (sh->a_structure != AS_A_DIAGONAL && sh->a_structure != AS_A_SCALAR) return AS_ERR_SHAPE;
   if (sh->io != AS_F32 && sh->io != AS_BF16) return AS_ERR_DTYPE;
   if (sh->d_model % 8 != 0) return AS_ERR_ALIGN;
   if (sh->batch > 65535) return AS_ERR_SHAPE;
@@ -150,7 +151,7 @@ int zero_outputs(const Plan& pl, uint32_t flags, const as_grads_t* out, char* ws
     AS_TRY((int)cudaMemsetAsync(out->db_delta, 0, P * 4, st));
     AS_TRY((int)cudaMemsetAsync(out->dW_B, 0, NS * P * 4, st));
     AS_TRY((int)cudaMemsetAsync(out->dW_C, 0, NS * P * 4, st));
-    AS_TRY((int)cudaMemsetAsync(out->dA_log, 0, P * NS * 4, st));
+    AS_TRY((int)cudaMemsetAsync(out->dA_log, 0, (pl.scalar ? P : P * NS) * 4, st));
   }
   return AS_OK;
 }

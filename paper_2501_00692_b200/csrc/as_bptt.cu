@@ -19,7 +19,7 @@ __global__ void bptt_forward_kernel(Plan pl, const IO* __restrict__ x, const flo
   float* snap = reinterpret_cast<float*>(ws + pl.off_bptt_ckpt);
   const int64_t nck = (pl.T + BCK - 1) / BCK;
   float A[NS], h[NS];
-  for (int n = 0; n < NS; ++n) { A[n] = -expf(A_log[(int64_t)p * NS + n]); h[n] = 0.f; }
+  for (int n = 0; n < NS; ++n) { A[n] = -expf(pl.scalar ? A_log[p] : A_log[(int64_t)p * NS + n]); h[n] = 0.f; }
   for (int64_t t = 0; t < pl.T; ++t) {
     if (t % BCK == 0)
       for (int n = 0; n < NS; ++n) snap[(((int64_t)b * nck + t / BCK) * pl.P + p) * NS + n] = h[n];
@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(32) bptt_reverse_kernel(Plan pl, const IO* __r
   float* dbc = reinterpret_cast<float*>(ws + pl.off_dbc);
   const int64_t nck = (pl.T + BCK - 1) / BCK;
   float A[NS], dh[NS], dA[NS];
-  for (int n = 0; n < NS; ++n) { A[n] = -expf(A_log[(int64_t)p * NS + n]); dh[n] = 0.f; dA[n] = 0.f; }
+  for (int n = 0; n < NS; ++n) { A[n] = -expf(pl.scalar ? A_log[p] : A_log[(int64_t)p * NS + n]); dh[n] = 0.f; dA[n] = 0.f; }
   float dbias = 0.f;
   float H[BCK + 1][NS];  // H[k] = state before token (chunk start + k)
   for (int64_t c = nck - 1; c >= 0; --c) {
@@ -97,7 +97,13 @@ __global__ void __launch_bounds__(32) bptt_reverse_kernel(Plan pl, const IO* __r
     }
   }
   if (active) {
-    for (int n = 0; n < NS; ++n) atomicAdd(dA_log + (int64_t)p * NS + n, dA[n] * A[n]);
+    if (pl.scalar) {
+      float tot = 0.f;
+      for (int n = 0; n < NS; ++n) tot += dA[n] * A[n];
+      atomicAdd(dA_log + p, tot);
+    } else {
+      for (int n = 0; n < NS; ++n) atomicAdd(dA_log + (int64_t)p * NS + n, dA[n] * A[n]);
+    }
     atomicAdd(db_delta + p, dbias);
   }
 }

@@ -61,6 +61,7 @@ struct Plan {
   int m;            // tbar / L   (whole segments inside a window that starts on a segment boundary)
   int r;            // tbar % L   (tokens of the following partial segment)
   int io;           // as_dtype_t
+  int scalar;       // 1: one decay rate per channel (A_log is [P]), 0: one per (channel, state)
   int tiles;        // ceil(P / CH) channel tiles
   int bw;           // channels per staged row: min(CH, P)
   int tc;           // 1: bf16 tensor-core contractions (bf16 I/O and d_model % 32 == 0), 0: FP32-pipe GEMMs

@@ -26,6 +26,7 @@ static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 int make_plan(const as_shape_t* sh, int64_t tbar, Plan* pl) {
   Plan p{};
   p.B = sh->batch; p.P = sh->d_model; p.T = sh->seqlen; p.io = sh->io;
+  p.scalar = sh->a_structure == AS_A_SCALAR ? 1 : 0;
   p.tc = (sh->io == AS_BF16 && sh->d_model % 32 == 0) ? 1 : 0;
   p.du_ld = p.tc ? p.P + NBC : p.P;
   p.full = tbar >= p.T;
@@ -229,11 +230,15 @@ __device__ __forceinline__ Who who(int tile, int P) {
   return w;
 }
 // A2[u] = -exp(A_log) * log2(e) for unit u = ch*4 + m  ->  states (8*half + 2m, +1) of channel pa + ch
-__device__ __forceinline__ void load_A2(const float* A_log, const Who& w, u64 (&A2)[NU]) {
+// (scalar structure: the channel's single rate for every state)
+__device__ __forceinline__ void load_A2(const float* A_log, const Who& w, u64 (&A2)[NU], int scalar) {
 #pragma unroll
   for (int u = 0; u < NU; ++u) {
     float2 v = make_float2(0.f, 0.f);
-    if (w.act) v = __ldg(reinterpret_cast<const float2*>(A_log + (int64_t)(w.pa + u / 4) * NS + 8 * w.half + 2 * (u % 4)));
+    if (w.act) {
+      if (scalar) { const float a = __ldg(A_log + w.pa + u / 4); v = make_float2(a, a); }
+      else v = __ldg(reinterpret_cast<const float2*>(A_log + (int64_t)(w.pa + u / 4) * NS + 8 * w.half + 2 * (u % 4)));
+    }
     A2[u] = pk(-__expf(v.x) * LOG2E, -__expf(v.y) * LOG2E);
   }
 }
@@ -333,7 +338,7 @@ __global__ void __launch_bounds__(NTHR) ascend_kernel(const __grid_constant__ CU
     for (int c = 0; c < NSTAGE && c < nchunk; ++c) issue(c);
 
   u64 A2[NU], h[NU], Pr[NU], acc[NU], snap[NU];
-  load_A2(A_log, w, A2);
+  load_A2(A_log, w, A2, pl.scalar);
   const int64_t sb = ((int64_t)b * pl.S + s) * pl.tiles + tile;
   if (MODE == PRE_Y) {
     load_block_g(reinterpret_cast<const float*>(ws + pl.off_hstart) + sb * TILE_FLOATS, w.tid, h);
@@ -466,7 +471,7 @@ __global__ void __launch_bounds__(NTHR) fixup_h_kernel(Plan pl, const float* __r
   const int tile = blockIdx.x, b = blockIdx.y;
   const Who w = who(tile, pl.P);
   u64 A2[NU], hs[NU];
-  load_A2(A_log, w, A2);
+  load_A2(A_log, w, A2, pl.scalar);
 #pragma unroll
   for (int u = 0; u < NU; ++u) hs[u] = 0ull;
   const float* hend = reinterpret_cast<const float*>(ws + pl.off_hend);
@@ -509,7 +514,7 @@ __global__ void __launch_bounds__(NTHR) fixup_mu_kernel(Plan pl, const float* __
   const int P = pl.P, S = pl.S;
   const Who w = who(tile, P);
   u64 A2[NU];
-  load_A2(A_log, w, A2);
+  load_A2(A_log, w, A2, pl.scalar);
   const float* muloc = reinterpret_cast<const float*>(ws + pl.off_muloc);
   const float* mupart = reinterpret_cast<const float*>(ws + pl.off_mupart);
   const float* segd = reinterpret_cast<const float*>(ws + pl.off_segd);
@@ -743,7 +748,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   }
 
   u64 A2[NU], mu[NU], dAacc[NU];
-  load_A2(A_log, w, A2);
+  load_A2(A_log, w, A2, pl.scalar);
   const int64_t sb = ((int64_t)b * pl.S + s) * pl.tiles + tile;
   load_block_g(reinterpret_cast<const float*>(ws + pl.off_carry) + sb * TILE_FLOATS, w.tid, mu);
   {   // true segment-start state: parked in shared memory
@@ -1012,7 +1017,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   if (failed) {
     if (w.tid == 0) atomicExch(status, AS_ERR_TIMEOUT);
   } else {
-    if (w.act) {
+    if (w.act && !pl.scalar) {
 #pragma unroll
       for (int u = 0; u < NU; ++u) {
         float alo, ahi, vlo, vhi;
@@ -1022,6 +1027,22 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         atomicAdd(dst, vlo * (alo * LN2));
         atomicAdd(dst + 1, vhi * (ahi * LN2));
       }
+    }
+    if (pl.scalar) {   // tied rate: the channel's gradient is the sum over its 16 states (8 here, 8 in the pair lane)
+      float tot[NCH];
+#pragma unroll
+      for (int ch = 0; ch < NCH; ++ch) {
+        tot[ch] = 0.f;
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+          float alo, ahi, vlo, vhi;
+          upk(A2[ch * 4 + m], alo, ahi);
+          upk(dAacc[ch * 4 + m], vlo, vhi);
+          tot[ch] += vlo * (alo * LN2) + vhi * (ahi * LN2);
+        }
+        tot[ch] += __shfl_xor_sync(0xffffffffu, tot[ch], 1);
+      }
+      if (fin) atomicAdd(dA_log + pmine, chf ? tot[NCH - 1] : tot[0]);
     }
     if (fin) atomicAdd(db_delta + pmine, dbacc);
   }

@@ -31,16 +31,16 @@ def test_exports_match_header(L):
 
 
 def test_version_and_strerror(L):
-    assert B.as_version() == 100
+    assert B.as_version() == 101
     assert B.strerror(0) == "ok"
     assert "tbar" in B.strerror(B.AS_ERR_TBAR)
     assert "unknown" in B.strerror(-999)
 
 
 def test_struct_layout_matches_c():
-    # int32, (pad), int64, 3 x int32, (pad)  ->  32 bytes with natural alignment
+    # int32, (pad), int64, 4 x int32  ->  32 bytes with natural alignment
     assert C.sizeof(B.as_shape_t) == 32
-    assert B.as_shape_t.seqlen.offset == 8 and B.as_shape_t.d_model.offset == 16
+    assert B.as_shape_t.seqlen.offset == 8 and B.as_shape_t.d_model.offset == 16 and B.as_shape_t.a_structure.offset == 28
     assert C.sizeof(B.as_params_t) == 40 and C.sizeof(B.as_grads_t) == 48
 
 
@@ -49,7 +49,8 @@ def test_workspace_query_and_argument_errors(L):
     fwd, grad = B.as_workspace_bytes(sh, 2048)
     assert 0 < fwd < grad < 8 << 30
     for bad, code in ((B.make_shape(0, 8, 64), B.AS_ERR_SHAPE), (B.make_shape(1, 8, 64, 8), B.AS_ERR_SHAPE),
-                      (B.make_shape(1, 8, 64, 16, 7), B.AS_ERR_DTYPE), (B.make_shape(1, 8, 60), B.AS_ERR_ALIGN)):
+                      (B.make_shape(1, 8, 64, 16, 7), B.AS_ERR_DTYPE), (B.make_shape(1, 8, 60), B.AS_ERR_ALIGN),
+                      (B.make_shape(1, 8, 64, 16, B.AS_F32, 5), B.AS_ERR_SHAPE)):
         with pytest.raises(B.AsError) as ei:
             B.as_workspace_bytes(bad, 4)
         assert ei.value.code == code

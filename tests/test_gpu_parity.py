@@ -154,3 +154,30 @@ def test_zero_upstream_gradient_gives_zero():
     g = gpu_adjoint(w, theta, x, dy, w.tbar)
     for k in O.PARAM_GRADS + ("dx",):
         assert float(g[k].abs().max()) == 0.0, k
+
+
+# ---- scalar structure: one decay rate per channel (Table 1 "Scalar SSM") ---------------------------------------------
+@pytest.mark.parametrize("io,T,P,tbar", [("f32", 700, 64, 700), ("f32", 1300, 136, 90), ("bf16", 2100, 256, 300),
+                                         ("bf16", 900, 96, 900)])
+def test_scalar_structure_matches_oracle(io, T, P, tbar):
+    w = synth.custom_workload("scalar", 21, 2, T, P, tbar=tbar, io=io)
+    theta, x, dy = setup(w, slow=True)
+    theta = dict(theta)
+    theta["A_log"] = theta["A_log"][:, 3].contiguous()            # [P]: the tied rate
+    sh = B.shape_of(x, w.d_state, a_scalar=True)
+    fb, gb = B.as_workspace_bytes(sh, tbar)
+    ws = B.alloc_workspace(gb, DEV)
+    grads = B.alloc_grads(sh, DEV)
+    assert tuple(grads["dA_log"].shape) == (P,)
+    y = torch.empty_like(x)
+    B.as_ssm_forward(sh, theta, x, y, ws)
+    B.as_adjoint_grad(sh, theta, x, dy, tbar, grads, ws)
+    assert B.as_check_status(ws) == 0
+    th = theta_f64(theta)
+    ref = O.batched(O.scalar_adjoint_grad, th, synth.to_f64(x), synth.to_f64(dy), tbar, w.d_state, tier="block")
+    compare_grads(grads, ref, TOL[io])
+    assert_close(synth.to_f64(y), ref["y"], TOL[io], "y")
+    if tbar >= T:   # the backpropagation comparator ties the rate the same way
+        gb2 = B.alloc_grads(sh, DEV)
+        B.as_full_bptt_grad(sh, theta, x, dy, gb2, ws)
+        compare_grads(gb2, ref, TOL[io])
