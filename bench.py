@@ -152,6 +152,7 @@ def main():
     ap.add_argument("--seq-len", type=int, default=None, help="override the workload's seqlen (profiling runs)")
     ap.add_argument("--tbar", type=int, default=None, help="override the workload's window (profiling runs)")
     ap.add_argument("--slow-decay", action="store_true", help="slow-decay parameter law (window term live)")
+    ap.add_argument("--scalar-a", action="store_true", help="scalar structure: one decay rate per channel (not the headline workload)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     if args.impl == "reference":
@@ -183,7 +184,10 @@ def main():
                                   w.d_model, w.d_state, 1, args.tbar or w.tbar, w.io)
     theta = synth.layer_params(w, 0, dev, slow_decay=args.slow_decay)
     x, dy = synth.activations(w, dev)
-    sh = B.shape_of(x, w.d_state)
+    if args.scalar_a:
+        theta = dict(theta)
+        theta["A_log"] = theta["A_log"][:, 0].contiguous()
+    sh = B.shape_of(x, w.d_state, a_scalar=args.scalar_a)
     _, gbytes = B.as_workspace_bytes(sh, w.tbar)
     ws = B.alloc_workspace(gbytes, dev)
     grads = B.alloc_grads(sh, dev)

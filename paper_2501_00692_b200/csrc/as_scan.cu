@@ -296,7 +296,7 @@ __device__ __forceinline__ void zero_rows(uint8_t* tile, int row_bytes, int nt, 
   for (int i = tid; i < n16; i += NTHR) p[i] = make_uint4(0u, 0u, 0u, 0u);
 }
 
-template <typename IO, int MODE>
+template <typename IO, int MODE, bool SC>
 __global__ void __launch_bounds__(NTHR) ascend_kernel(const __grid_constant__ CUtensorMap tmX,
                                                     const __grid_constant__ CUtensorMap tmD,
                                                     const __grid_constant__ CUtensorMap tmG, Plan pl,
@@ -396,10 +396,12 @@ __global__ void __launch_bounds__(NTHR) ascend_kernel(const __grid_constant__ CU
           const u64 d2 = pk(ddc, ddc), dx2 = pk(dxc, dxc), g2 = pk(gc, gc);
           yv[ch] = 0.f;
           u64 yacc = 0ull;
+          u64 ach = 0ull;
+          if (SC) ach = ex2_2(mul2(d2, A2[ch * 4]));   // scalar rate: one factor for the channel's states
 #pragma unroll
           for (int m = 0; m < 4; ++m) {
             const int u = ch * 4 + m;
-            const u64 a = ex2_2(mul2(d2, A2[u]));
+            const u64 a = SC ? ach : ex2_2(mul2(d2, A2[u]));
             h[u] = fma2(a, h[u], mul2(dx2, Bp[m]));
             if (MU) {
               Pr[u] = mul2(Pr[u], a);
@@ -573,6 +575,23 @@ __global__ void __launch_bounds__(NTHR) fixup_mu_kernel(Plan pl, const float* __
   }
 }
 
+// abar for the NU units of a thread from the per-channel exponent scale e2[ch] = {e, e}: exp2(e * A2[u]).  With a
+// scalar rate the N states of a channel share one factor, so one pair of MUFU operations per channel is enough.
+template <bool SC>
+__device__ __forceinline__ void decay_units(const u64 (&e2)[NCH], const u64 (&A2)[NU], u64 (&a)[NU]) {
+  if (SC) {
+#pragma unroll
+    for (int ch = 0; ch < NCH; ++ch) {
+      const u64 ac = ex2_2(mul2(e2[ch], A2[ch * 4]));
+#pragma unroll
+      for (int m = 0; m < 4; ++m) a[ch * 4 + m] = ac;
+    }
+  } else {
+#pragma unroll
+    for (int u = 0; u < NU; ++u) a[u] = ex2_2(mul2(e2[u / 4], A2[u]));
+  }
+}
+
 // ---- tensor memory as a per-thread scratchpad ------------------------------------------------------
 // The main adjoint kernel runs no MMA, so the SM's tensor memory is free.  Each CTA allocates 128 of the 512
 // columns of its SM (three CTAs are resident) and every thread parks the chunk's eight states in its own TMEM lane:
@@ -647,7 +666,7 @@ template <int ESZ, bool WIN> struct MainCfg {
 // then walk the chunk's tokens backwards: mu recurrence (with the exact window exit), the per-token
 // vector-Jacobian products, the channel sums dB_t / dC_t, and the per-channel outputs du_t and dx_dir_t.
 // ------------------------------------------------------------------------------------------------
-template <typename IO, bool FULL>
+template <typename IO, bool FULL, bool SC>
 __global__ void __launch_bounds__(NTHR, MAIN_CTAS)
 adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmD,
                     const __grid_constant__ CUtensorMap tmG, Plan pl, const float* __restrict__ A_log,
@@ -822,8 +841,10 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
           if (!w.act) csv = 0.f;   // the 1D copy only covers existing channels
           c2[c] = pk(csv, csv);
         }
+        u64 dec[NU];
+        decay_units<SC>(c2, A2, dec);
 #pragma unroll
-        for (int u = 0; u < NU; ++u) h[u] = fma2(ex2_2(mul2(c2[u / 4], A2[u])), hst[u], h[u]);
+        for (int u = 0; u < NU; ++u) h[u] = fma2(dec[u], hst[u], h[u]);
       }
       if (WIN) {
         // Delta of the tokens leaving the window during this chunk.  Inside the chunk the window sum never drops
@@ -858,8 +879,10 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
             const float dxc = dv.v[c] * xv.v[c];
             d2[c] = pk(dv.v[c], dv.v[c]); dx2[c] = pk(dxc, dxc);
           }
+          u64 af[NU];
+          decay_units<SC>(d2, A2, af);
 #pragma unroll
-          for (int u = 0; u < NU; ++u) h[u] = fma2(ex2_2(mul2(d2[u / 4], A2[u])), h[u], mul2(dx2[u / 4], Bp[u % 4]));
+          for (int u = 0; u < NU; ++u) h[u] = fma2(af[u], h[u], mul2(dx2[u / 4], Bp[u % 4]));
           tmem_st16(tm + 16 * j, h);
         }
         tmem_wait_st();
@@ -926,19 +949,22 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
             sw2[c] = pk(swf, swf);
             swl[c] += dd[c] - d2v.v[c] * wm;   // window of token t-1: (t-1, t-1+Tbar]
           }
+          u64 wf[NU];
+          decay_units<SC>(sw2, A2, wf);
 #pragma unroll
-          for (int u = 0; u < NU; ++u)
-            mu[u] = fma2(ex2_2(mul2(sw2[u / 4], A2[u])), mul2(ng2[u / 4], C2p[u % 4]), mu[u]);
+          for (int u = 0; u < NU; ++u) mu[u] = fma2(wf[u], mul2(ng2[u / 4], C2p[u % 4]), mu[u]);
         }
         u64 vB[4], vC[4];
         float ssum[NCH], dsum[NCH];
 #pragma unroll
         for (int ch = 0; ch < NCH; ++ch) {
           u64 sacc, dacc;
+          u64 ach = 0ull;
+          if (SC) ach = ex2_2(mul2(d2[ch], A2[ch * 4]));   // scalar rate: one factor for the channel's states
 #pragma unroll
           for (int m = 0; m < 4; ++m) {
             const int u = ch * 4 + m;
-            const u64 a = ex2_2(mul2(d2[ch], A2[u]));
+            const u64 a = SC ? ach : ex2_2(mul2(d2[ch], A2[u]));
             const u64 hn = hT[u];                                  // h_i
             const u64 hb = fma2(ndx2[ch], Bp[m], hn);              // abar_i h_{i-1} = h_i - Delta_i x_i B_i
             vB[m] = ch == 0 ? mul2(mu[u], dx2[ch]) : fma2(mu[u], dx2[ch], vB[m]);   // dB partial (two channels)
@@ -1117,13 +1143,13 @@ int set_smem(K kern, int bytes) {
   return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess ? 0 : 1;
 }
 
-template <typename IO, int MODE>
+template <typename IO, int MODE, bool SC>
 int launch_ascend_t(const Plan& pl, const ScanPtrs& sp, void* y, cudaStream_t st) {
   Maps m;
   if (make_maps(pl, sp, &m)) return 1;
   using St = Stage<sizeof(IO), MODE == PRE_ADJ, false, false>;
   const int bytes = NSTAGE * St::BYTES + 128;
-  auto kern = ascend_kernel<IO, MODE>;
+  auto kern = ascend_kernel<IO, MODE, SC>;
   static bool once = false;
   if (!once) { if (set_smem(kern, bytes)) return 1; once = true; }
   kern<<<dim3(pl.tiles, pl.S, pl.B), NTHR, bytes, st>>>(m.x, m.d, m.g, pl, sp.A_log, sp.ws, (IO*)y);
@@ -1131,12 +1157,12 @@ int launch_ascend_t(const Plan& pl, const ScanPtrs& sp, void* y, cudaStream_t st
   return (int)cudaGetLastError();
 }
 
-template <typename IO, bool FULL>
+template <typename IO, bool FULL, bool SC>
 int launch_main_t(const Plan& pl, const ScanPtrs& sp, float* dA_log, float* db_delta, cudaStream_t st) {
   Maps m;
   if (make_maps(pl, sp, &m)) return 1;
   const int bytes = MainCfg<sizeof(IO), !FULL>::SMEM_DYN;
-  auto kern = adjoint_main_kernel<IO, FULL>;
+  auto kern = adjoint_main_kernel<IO, FULL, SC>;
   static bool once = false;
   if (!once) { if (set_smem(kern, bytes)) return 1; once = true; }
   kern<<<dim3(pl.tiles, pl.S, pl.B), NTHR, bytes, st>>>(m.x, m.d, m.g, pl, sp.A_log, sp.ws, dA_log, db_delta);
@@ -1149,11 +1175,21 @@ int launch_main_t(const Plan& pl, const ScanPtrs& sp, float* dA_log, float* db_d
 // ------------------------------------------------------------------------------------------------
 // launchers
 // ------------------------------------------------------------------------------------------------
+template <typename IO, int MODE>
+int launch_ascend_s(const Plan& pl, const ScanPtrs& sp, void* y, cudaStream_t st) {
+  return pl.scalar ? launch_ascend_t<IO, MODE, true>(pl, sp, y, st) : launch_ascend_t<IO, MODE, false>(pl, sp, y, st);
+}
+template <typename IO, bool FULL>
+int launch_main_s(const Plan& pl, const ScanPtrs& sp, float* dA_log, float* db_delta, cudaStream_t st) {
+  return pl.scalar ? launch_main_t<IO, FULL, true>(pl, sp, dA_log, db_delta, st)
+                   : launch_main_t<IO, FULL, false>(pl, sp, dA_log, db_delta, st);
+}
+
 int launch_prepass(const Plan& pl, const ScanPtrs& sp, bool with_mu, cudaStream_t st) {
   if (pl.io == AS_BF16)
-    return with_mu ? launch_ascend_t<__nv_bfloat16, PRE_ADJ>(pl, sp, nullptr, st)
-                   : launch_ascend_t<__nv_bfloat16, PRE_FWD>(pl, sp, nullptr, st);
-  return with_mu ? launch_ascend_t<float, PRE_ADJ>(pl, sp, nullptr, st) : launch_ascend_t<float, PRE_FWD>(pl, sp, nullptr, st);
+    return with_mu ? launch_ascend_s<__nv_bfloat16, PRE_ADJ>(pl, sp, nullptr, st)
+                   : launch_ascend_s<__nv_bfloat16, PRE_FWD>(pl, sp, nullptr, st);
+  return with_mu ? launch_ascend_s<float, PRE_ADJ>(pl, sp, nullptr, st) : launch_ascend_s<float, PRE_FWD>(pl, sp, nullptr, st);
 }
 
 int launch_fixup(const Plan& pl, const ScanPtrs& sp, bool with_mu, cudaStream_t st) {
@@ -1167,16 +1203,16 @@ int launch_fixup(const Plan& pl, const ScanPtrs& sp, bool with_mu, cudaStream_t 
 }
 
 int launch_forward_y(const Plan& pl, const ScanPtrs& sp, void* y, cudaStream_t st) {
-  if (pl.io == AS_BF16) return launch_ascend_t<__nv_bfloat16, PRE_Y>(pl, sp, y, st);
-  return launch_ascend_t<float, PRE_Y>(pl, sp, y, st);
+  if (pl.io == AS_BF16) return launch_ascend_s<__nv_bfloat16, PRE_Y>(pl, sp, y, st);
+  return launch_ascend_s<float, PRE_Y>(pl, sp, y, st);
 }
 
 int launch_adjoint_main(const Plan& pl, const ScanPtrs& sp, float* dA_log, float* db_delta, cudaStream_t st) {
   if (pl.io == AS_BF16)
-    return pl.full ? launch_main_t<__nv_bfloat16, true>(pl, sp, dA_log, db_delta, st)
-                   : launch_main_t<__nv_bfloat16, false>(pl, sp, dA_log, db_delta, st);
-  return pl.full ? launch_main_t<float, true>(pl, sp, dA_log, db_delta, st)
-                 : launch_main_t<float, false>(pl, sp, dA_log, db_delta, st);
+    return pl.full ? launch_main_s<__nv_bfloat16, true>(pl, sp, dA_log, db_delta, st)
+                   : launch_main_s<__nv_bfloat16, false>(pl, sp, dA_log, db_delta, st);
+  return pl.full ? launch_main_s<float, true>(pl, sp, dA_log, db_delta, st)
+                 : launch_main_s<float, false>(pl, sp, dA_log, db_delta, st);
 }
 
 int launch_wait_selftest(int* status, unsigned limit, cudaStream_t st) {
