@@ -145,23 +145,18 @@ __device__ __forceinline__ void bulk_1d(void* dst, const void* src, uint32_t byt
 
 template <typename IO> struct IoSz { static constexpr int v = sizeof(IO); };
 
-// shared-memory stage of one chunk
-template <int ESZ, bool WITH_G, bool WITH_CKPT, bool WIN>
+// shared-memory stage of one chunk of the ascending kernels: x, Delta, [B | C] rows and (pre-pass) dy
+template <int ESZ, bool WITH_G>
 struct Stage {
   static constexpr int X = 0;
   static constexpr int D = X + CK * CH * ESZ;
   static constexpr int BC = D + CK * CH * 4;
   static constexpr int G = BC + CK * NBC * 4;
-  static constexpr int CKP = G + (WITH_G ? CK * CH * ESZ : 0);
-  static constexpr int CS = CKP + (WITH_CKPT ? TILE_FLOATS * 4 : 0);
-  static constexpr int G2 = CS + (WITH_CKPT ? CH * 4 : 0);
-  static constexpr int D2 = G2 + (WIN ? CK * CH * ESZ : 0);
-  static constexpr int BC2 = D2 + (WIN ? CK * CH * 4 : 0);
-  static constexpr int BYTES = BC2 + (WIN ? CK * NBC * 4 : 0);
+  static constexpr int BYTES = G + (WITH_G ? CK * CH * ESZ : 0);
 };
 constexpr int NSTAGE = 3;        // ascending kernels
 constexpr int WRED_Q = 32 * 4 + 8;   // floats per quarter-block of the per-warp reduction scratch (512 B + 32 B skew)
-constexpr int MAIN_CTAS = 3;    // resident CTAs per SM the main kernel is compiled for (168 registers per thread)
+constexpr int MAIN_CTAS = 3;    // resident CTAs per SM the main kernel is compiled for (up to 168 registers per thread)
 constexpr int BW_UNROLL = 4;     // unroll factor of the main adjoint kernel's backward token loop
 constexpr int NSTAGE_MAIN = 2;   // main adjoint kernel: a chunk takes thousands of cycles, one chunk of lookahead suffices
 
@@ -304,7 +299,7 @@ __global__ void __launch_bounds__(NTHR) ascend_kernel(const __grid_constant__ CU
                                                     IO* __restrict__ y) {
   constexpr int ESZ = IoSz<IO>::v;
   constexpr bool MU = MODE == PRE_ADJ;
-  using St = Stage<ESZ, MU, false, false>;
+  using St = Stage<ESZ, MU>;
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[NSTAGE];
   uint8_t* smem = smem_raw + ((128u - (smem_u32(smem_raw) & 127u)) & 127u);   // stays a shared-space pointer
@@ -1147,7 +1142,7 @@ template <typename IO, int MODE, bool SC>
 int launch_ascend_t(const Plan& pl, const ScanPtrs& sp, void* y, cudaStream_t st) {
   Maps m;
   if (make_maps(pl, sp, &m)) return 1;
-  using St = Stage<sizeof(IO), MODE == PRE_ADJ, false, false>;
+  using St = Stage<sizeof(IO), MODE == PRE_ADJ>;
   const int bytes = NSTAGE * St::BYTES + 128;
   auto kern = ascend_kernel<IO, MODE, SC>;
   static bool once = false;
