@@ -461,12 +461,9 @@ int make_map_out_bf16(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t
 
 template <int AMAJ, int BMAJ, int EPI, int BN>
 int launch_tc(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap (&tmO)[3], const TcArgs& a, cudaStream_t st) {
-  static bool attr_set = false;
   auto kern = gemm_tc_kernel<AMAJ, BMAJ, EPI, BN>;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::SMEM_DYN) != cudaSuccess) return 1;
-    attr_set = true;
-  }
+  static bool done[AS_MAX_DEVICES] = {};
+  if (ensure_dynamic_smem(kern, Cfg<BN>::SMEM_DYN, done)) return 1;
   const int64_t ntiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN) * a.splitk;
   const unsigned grid = (unsigned)(ntiles < 148 ? ntiles : 148);   // one persistent CTA per SM
   kern<<<grid, NTHREADS, Cfg<BN>::SMEM_DYN, st>>>(tmA, tmB, tmO[0], tmO[1], tmO[2], a);

@@ -15,6 +15,20 @@ namespace as {
 extern std::atomic<int64_t> g_launches;   // kernels launched by this library (diagnostic)
 inline void count_launch(int n = 1) { g_launches.fetch_add(n); }
 
+// Function attributes (the dynamic shared-memory limit) belong to a device: remember per device, per kernel
+// instantiation, whether the limit has been raised.  `done` is a static array of the launcher, one flag per device.
+constexpr int AS_MAX_DEVICES = 64;
+template <typename K>
+inline int ensure_dynamic_smem(K kern, int bytes, bool (&done)[AS_MAX_DEVICES]) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= AS_MAX_DEVICES) return 1;
+  if (!done[dev]) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return 1;
+    done[dev] = true;
+  }
+  return 0;
+}
+
 constexpr int NS = 16;        // d_state handled by the scan kernels
 constexpr int CK = 8;         // tokens per checkpoint chunk (h of one chunk lives in registers)
 constexpr int NCH = 2;        // channels per thread of the scan kernels (1 or 2)

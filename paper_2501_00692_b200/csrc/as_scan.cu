@@ -1135,10 +1135,6 @@ int make_maps(const Plan& pl, const ScanPtrs& sp, Maps* m) {
   return 0;
 }
 
-template <typename K>
-int set_smem(K kern, int bytes) {
-  return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess ? 0 : 1;
-}
 
 template <typename IO, int MODE, bool SC>
 int launch_ascend_t(const Plan& pl, const ScanPtrs& sp, void* y, cudaStream_t st) {
@@ -1147,8 +1143,8 @@ int launch_ascend_t(const Plan& pl, const ScanPtrs& sp, void* y, cudaStream_t st
   using St = Stage<sizeof(IO), MODE == PRE_ADJ>;
   const int bytes = NSTAGE * St::BYTES + 128;
   auto kern = ascend_kernel<IO, MODE, SC>;
-  static bool once = false;
-  if (!once) { if (set_smem(kern, bytes)) return 1; once = true; }
+  static bool done[AS_MAX_DEVICES] = {};
+  if (ensure_dynamic_smem(kern, bytes, done)) return 1;
   kern<<<dim3(pl.tiles, pl.S, pl.B), NTHR, bytes, st>>>(m.x, m.d, m.g, pl, sp.A_log, sp.ws, (IO*)y);
   count_launch();
   return (int)cudaGetLastError();
@@ -1160,8 +1156,8 @@ int launch_main_t(const Plan& pl, const ScanPtrs& sp, float* dA_log, float* db_d
   if (make_maps(pl, sp, &m)) return 1;
   const int bytes = MainCfg<sizeof(IO), !FULL>::SMEM_DYN;
   auto kern = adjoint_main_kernel<IO, FULL, SC>;
-  static bool once = false;
-  if (!once) { if (set_smem(kern, bytes)) return 1; once = true; }
+  static bool done[AS_MAX_DEVICES] = {};
+  if (ensure_dynamic_smem(kern, bytes, done)) return 1;
   kern<<<dim3(pl.tiles, pl.S, pl.B), NTHR, bytes, st>>>(m.x, m.d, m.g, pl, sp.A_log, sp.ws, dA_log, db_delta);
   count_launch();
   return (int)cudaGetLastError();
