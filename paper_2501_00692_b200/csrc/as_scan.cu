@@ -157,7 +157,8 @@ struct Stage {
 constexpr int NSTAGE = 3;        // ascending kernels
 constexpr int WRED_Q = 32 * 4 + 8;   // floats per quarter-block of the per-warp reduction scratch (512 B + 32 B skew)
 constexpr int MAIN_CTAS = 3;    // resident CTAs per SM the main kernel is compiled for (up to 168 registers per thread)
-constexpr int BW_UNROLL = 4;     // unroll factor of the main adjoint kernel's backward token loop
+constexpr int FW_UNROLL = 4;     // unroll factor of the main adjoint kernel's forward rebuild loop
+constexpr int BW_UNROLL = 2;     // unroll factor of the main adjoint kernel's backward token loop
 constexpr int NSTAGE_MAIN = 2;   // main adjoint kernel: a chunk takes thousands of cycles, one chunk of lookahead suffices
 
 // per-thread values of its NCH channels
@@ -675,7 +676,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   __shared__ __align__(8) uint64_t ckp_bar;          // the checkpoint tile of the current chunk has landed
   __shared__ __align__(8) uint64_t ckp_free;         // all threads have read it (NTHR arrivals)
   __shared__ uint32_t tmem_base_s;
-  __shared__ float red[2][CK][NBC];                 // per-token [dB | dC] sums of the CTA, two chunks in flight
+  __shared__ float red[2][NTHR / 32][CK][NBC];      // per-token [dB | dC] sums of each warp, two chunks in flight
   __shared__ __align__(16) float wred[NTHR / 32][4 * WRED_Q];   // per-warp scratch of the channel reduction
   __shared__ ulonglong2 hst_s[2 * NCH][NTHR];       // true segment-start state, read back once per chunk
   uint8_t* smem = smem_raw + ((128u - (smem_u32(smem_raw) & 127u)) & 127u);   // stays a shared-space pointer
@@ -719,7 +720,6 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  for (int e = w.tid; e < 2 * CK * NBC; e += NTHR) (&red[0][0][0])[e] = 0.f;
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -860,7 +860,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
       // forward rebuild: the states after the chunk's eight tokens go to tensor memory
       {
         const float* bck = reinterpret_cast<const float*>(sm + St::BC) + 8 * w.half;
-#pragma unroll 1
+#pragma unroll FW_UNROLL
         for (int j = 0; j < CK; ++j) {
           const ChV dv = lds_ch<float>(sm + St::D, j, w.k);
           const ChV xv = lds_ch<IO>(sm + St::X, j, w.k);
@@ -895,7 +895,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
       const uint8_t* pD = sm + St::D + (CK - 1) * CH * 4 + 4 * NCH * w.k;       // Delta row (fp32)
       const uint8_t* pX = sm + St::X + (CK - 1) * CH * ESZ + ESZ * NCH * w.k;   // x row; dy row at + (St::G - St::X)
       const float* pB = reinterpret_cast<const float*>(sm + St::BC) + 8 * w.half + (CK - 1) * NBC;   // [B | C] row
-      float* pR = &red[rb][CK - 1][((lane >> 1) & 8) * 2 + 8 * w.half + ((lane >> 1) & 7)];
+      float* pR = &red[rb][warp][CK - 1][((lane >> 1) & 8) * 2 + 8 * w.half + ((lane >> 1) & 7)];
       uint32_t tmj = tm + 16 * (CK - 1);
 #pragma unroll BW_UNROLL
       for (int j = CK - 1; j >= 0; --j) {
@@ -1016,8 +1016,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
           for (int wdt = 8; wdt >= 1; wdt >>= 1)   // pairwise tree: 4 dependent adds instead of 16
 #pragma unroll
             for (int i2 = 0; i2 < wdt; ++i2) part[i2] += part[i2 + wdt];
-          const float tot = part[0];
-          atomicAdd(pR, tot);
+          *pR = part[0];   // this warp's slot: plain store, the four warps are added up when the chunk is flushed
         }
         pD -= CH * 4; pX -= CH * ESZ; pB -= NBC; pR -= NBC;
       }
@@ -1032,8 +1031,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     if (w.tid == 0 && i + NSTAGE_MAIN < nchunk) issue(i + NSTAGE_MAIN);
     for (int e = w.tid; e < CK * NBC; e += NTHR) {
       const int j = e / NBC, q = e % NBC;
-      const float sum = red[rb][j][q];
-      red[rb][j][q] = 0.f;   // ready for the chunk after next
+      const float sum = (red[rb][0][j][q] + red[rb][1][j][q]) + (red[rb][2][j][q] + red[rb][3][j][q]);
       if (j < nt) atomicAdd(dbc + ((int64_t)b * T + tc + j) * NBC + q, sum);
     }
   }
