@@ -18,7 +18,7 @@ from . import binding as B
 
 class Stack:
     def __init__(self, thetas, batch, seqlen, d_model, d_state=16, dtype=torch.float32, device="cuda:0", tbar=None,
-                 eps=1e-6):
+                 eps=1e-6, paper_streams=1):
         self.thetas = thetas
         self.K = len(thetas)
         self.eps = eps
@@ -30,6 +30,10 @@ class Stack:
         self.ys = None       # y_0 .. y_K
         self.yhat = torch.empty(batch, seqlen, d_model, dtype=dtype, device=device)
         self.ytilde = torch.empty_like(self.yhat)
+        # "paper" mode only: the layers are independent, so they may run on several streams at once (the layer
+        # dimension of Section 4.2); every extra stream owns a workspace and a normalised-input buffer
+        self.extra = [(torch.cuda.Stream(device=device), B.alloc_workspace(gbytes, device), torch.empty_like(self.yhat))
+                      for _ in range(max(0, paper_streams - 1))]
 
     def forward(self, y0: torch.Tensor):
         """Runs the stack, keeping y_0..y_K (the per-layer inputs are re-normalised in the backward)."""
@@ -48,6 +52,8 @@ class Stack:
         assert self.ys is not None, "call forward() first"
         dev = g.device
         grads = [None] * self.K
+        if mode == "paper" and self.extra and record is None:
+            return self._paper_grad_concurrent(g), None
         G = g.clone() if mode == "chained" else g
         for k in range(self.K - 1, -1, -1):
             B.as_rmsnorm_fwd(self.shape, self.ys[k], self.yhat, self.eps)
@@ -60,3 +66,21 @@ class Stack:
                 gk["dx"] = None
             grads[k] = gk
         return grads, (G if mode == "chained" else None)
+
+    def _paper_grad_concurrent(self, g: torch.Tensor):
+        """Proposition 3 with the layers spread round-robin over the stack's streams."""
+        main = torch.cuda.current_stream()
+        lanes = [(main, self.ws, self.yhat)] + self.extra
+        for st, _, _ in self.extra:
+            st.wait_stream(main)
+        grads = [None] * self.K
+        for k in range(self.K - 1, -1, -1):
+            st, ws, yhat = lanes[k % len(lanes)]
+            with torch.cuda.stream(st):
+                B.as_rmsnorm_fwd(self.shape, self.ys[k], yhat, self.eps)
+                gk = B.alloc_grads(self.shape, g.device, with_dx=False)
+                B.as_adjoint_grad(self.shape, self.thetas[k], yhat, g, self.tbar, gk, ws)
+            grads[k] = gk
+        for st, _, _ in self.extra:
+            main.wait_stream(st)
+        return grads

@@ -65,6 +65,27 @@ def test_stack_gradients(io, K, T, P, tbar, mode):
         assert errors(synth.to_f64(G0), np.stack(G0all))[0] <= e2e
 
 
+def test_paper_mode_on_two_streams_equals_one_stream():
+    """Prop. 3's layers are independent: spreading them over two streams (each with its own workspace) changes nothing
+    but the order of the fp32 atomic sums."""
+    K, T, P, tbar = 6, 1200, 128, 256
+    w = synth.custom_workload("stack2", 5, 2, T, P, layers=K, tbar=tbar, io="bf16")
+    thetas = [synth.layer_params(w, k, DEV, slow_decay=True) for k in range(K)]
+    y0, g = synth.activations(w, DEV)
+    out = []
+    for ns in (1, 2):
+        st = Stack(thetas, w.batch, T, P, dtype=w.torch_dtype, device=DEV, tbar=tbar, paper_streams=ns)
+        st.forward(y0)
+        grads, _ = st.adjoint_grad(g, "paper")
+        torch.cuda.synchronize()
+        assert B.as_check_status(st.ws) == B.AS_OK
+        out.append(grads)
+    for a, b in zip(*out):
+        for k in O.PARAM_GRADS:
+            scale = float(a[k].abs().max())
+            assert float((a[k] - b[k]).abs().max()) <= 1e-2 * scale, k
+
+
 def test_c3_full_size_bf16():
     """Workload C3 in the launch configuration the benchmark times, every output against the oracle."""
     w = synth.WORKLOADS["C3"]
