@@ -410,12 +410,20 @@ __global__ void pack_wcat_kernel(int P, const __nv_bfloat16* __restrict__ Wd, co
   out[i] = row < P ? Wd[i] : (row < P + NS ? WB[(row - P) * P + col] : WC[(row - P - NS) * P + col]);
 }
 
+// [dB | dC] fp32 sums -> the last 32 bf16 columns of Gcat; eight values per thread (P and the row pitch are multiples
+// of 32 elements on this path, so every access is 16-byte aligned)
 __global__ void cvt_dbc_kernel(int64_t rows, int ldg, int P, const float* __restrict__ dbc, __nv_bfloat16* __restrict__ gcat) {
-  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= rows * NBC) return;
-  const int64_t row = i / NBC;
-  const int c = (int)(i % NBC);
-  gcat[row * ldg + P + c] = __float2bfloat16_rn(dbc[i]);
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;   // one group of 8 columns
+  if (i >= rows * (NBC / 8)) return;
+  const int64_t row = i / (NBC / 8);
+  const int c = (int)(i % (NBC / 8)) * 8;
+  const float4 a = __ldg(reinterpret_cast<const float4*>(dbc + row * NBC + c));
+  const float4 b = __ldg(reinterpret_cast<const float4*>(dbc + row * NBC + c + 4));
+  uint4 o;
+  __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&o);
+  o2[0] = __floats2bfloat162_rn(a.x, a.y); o2[1] = __floats2bfloat162_rn(a.z, a.w);
+  o2[2] = __floats2bfloat162_rn(b.x, b.y); o2[3] = __floats2bfloat162_rn(b.z, b.w);
+  *reinterpret_cast<uint4*>(gcat + row * ldg + P + c) = o;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -505,7 +513,7 @@ int tc_projections(const Plan& pl, const as_params_t* pr, const void* x, char* w
 int tc_weight_grads(const Plan& pl, const void* x, const as_grads_t* out, char* ws, cudaStream_t st) {
   const int64_t M = (int64_t)pl.B * pl.T;
   const int P = pl.P, NW = P + NBC;
-  cvt_dbc_kernel<<<(unsigned)((M * NBC + 255) / 256), 256, 0, st>>>(M, NW, P, (const float*)(ws + pl.off_dbc),
+  cvt_dbc_kernel<<<(unsigned)((M * (NBC / 8) + 255) / 256), 256, 0, st>>>(M, NW, P, (const float*)(ws + pl.off_dbc),
                                                                     (__nv_bfloat16*)(ws + pl.off_du));
   count_launch();
   if (cudaGetLastError() != cudaSuccess) return 1;

@@ -476,16 +476,19 @@ __global__ void __launch_bounds__(NTHR) fixup_h_kernel(Plan pl, const float* __r
   const float* segd = reinterpret_cast<const float*>(ws + pl.off_segd);
   float* hstart = reinterpret_cast<float*>(ws + pl.off_hstart);
   constexpr int UN = 4;
-  for (int s0 = 0; s0 < pl.S; s0 += UN) {
-    u64 he[UN][NU];
-    ChV sd[UN];
+  // software-pipelined over batches of UN segments: the loads of the next batch are in flight while this one is applied
+  u64 he[2][UN][NU];
+  ChV sd[2][UN];
+  auto fetch = [&](int s0, int buf) {
 #pragma unroll
     for (int i = 0; i < UN; ++i) {
       const int s = min(s0 + i, pl.S - 1);
       const int64_t sb = ((int64_t)b * pl.S + s) * pl.tiles + tile;
-      load_block_g(hend + sb * TILE_FLOATS, w.tid, he[i]);
-      sd[i] = w.act ? ldg_ch(segd + ((int64_t)b * pl.S + s) * pl.P + w.pa) : ch_zero();
+      load_block_g(hend + sb * TILE_FLOATS, w.tid, he[buf][i]);
+      sd[buf][i] = w.act ? ldg_ch(segd + ((int64_t)b * pl.S + s) * pl.P + w.pa) : ch_zero();
     }
+  };
+  auto apply = [&](int s0, int buf) {
 #pragma unroll
     for (int i = 0; i < UN; ++i) {
       const int s = s0 + i;
@@ -494,10 +497,19 @@ __global__ void __launch_bounds__(NTHR) fixup_h_kernel(Plan pl, const float* __r
         store_block(hstart + sb * TILE_FLOATS, w.tid, hs);
         u64 d2[NCH];
 #pragma unroll
-        for (int c = 0; c < NCH; ++c) d2[c] = pk(sd[i].v[c], sd[i].v[c]);
+        for (int c = 0; c < NCH; ++c) d2[c] = pk(sd[buf][i].v[c], sd[buf][i].v[c]);
 #pragma unroll
-        for (int u = 0; u < NU; ++u) hs[u] = fma2(ex2_2(mul2(d2[u / 4], A2[u])), hs[u], he[i][u]);
+        for (int u = 0; u < NU; ++u) hs[u] = fma2(ex2_2(mul2(d2[u / 4], A2[u])), hs[u], he[buf][i][u]);
       }
+    }
+  };
+  fetch(0, 0);
+  for (int s0 = 0; s0 < pl.S; s0 += 2 * UN) {
+    if (s0 + UN < pl.S) fetch(s0 + UN, 1);
+    apply(s0, 0);
+    if (s0 + UN < pl.S) {
+      if (s0 + 2 * UN < pl.S) fetch(s0 + 2 * UN, 0);
+      apply(s0 + UN, 1);
     }
   }
 }
