@@ -464,42 +464,44 @@ __global__ void __launch_bounds__(NTHR) ascend_kernel(const __grid_constant__ CU
 // ------------------------------------------------------------------------------------------------
 // carries across segments.  Thread (b, tile, tid) owns the same 16 (channel, state) slots as in the scans.
 // ------------------------------------------------------------------------------------------------
-// hstart[s]: true state entering segment s (sequential in s).
+// hstart[s]: true state entering segment s (sequential in s).  The recurrence over segments is a chain of dependent
+// steps, so the kernel is latency-bound: one thread per state pair (blockIdx.z = the unit u of the scan kernels'
+// thread), and the loads of a batch of 16 segments are issued together, one batch ahead of the one being applied.
 __global__ void __launch_bounds__(NTHR) fixup_h_kernel(Plan pl, const float* __restrict__ A_log, char* __restrict__ ws) {
-  const int tile = blockIdx.x, b = blockIdx.y;
+  const int tile = blockIdx.x, b = blockIdx.y, u = blockIdx.z;
   const Who w = who(tile, pl.P);
-  u64 A2[NU], hs[NU];
-  load_A2(A_log, w, A2, pl.scalar);
+  u64 A2all[NU];
+  load_A2(A_log, w, A2all, pl.scalar);
+  u64 A2u = 0ull;
 #pragma unroll
-  for (int u = 0; u < NU; ++u) hs[u] = 0ull;
-  const float* hend = reinterpret_cast<const float*>(ws + pl.off_hend);
+  for (int i = 0; i < NU; ++i) A2u = i == u ? A2all[i] : A2u;
+  const int ch = u / 4;                                  // which of the thread's channels the unit belongs to
+  const u64* hend = reinterpret_cast<const u64*>(ws + pl.off_hend);
   const float* segd = reinterpret_cast<const float*>(ws + pl.off_segd);
-  float* hstart = reinterpret_cast<float*>(ws + pl.off_hstart);
-  constexpr int UN = 4;
-  // software-pipelined over batches of UN segments: the loads of the next batch are in flight while this one is applied
-  u64 he[2][UN][NU];
-  ChV sd[2][UN];
+  u64* hstart = reinterpret_cast<u64*>(ws + pl.off_hstart);
+  // unit u of thread tid inside a tile block: float4 q = u / 2 at (q * NTHR + tid), its low or high half
+  const int64_t in_blk = ((int64_t)(u >> 1) * NTHR + w.tid) * 2 + (u & 1);   // in u64 units
+  constexpr int UN = 16;
+  u64 he[2][UN];
+  float sd[2][UN];
   auto fetch = [&](int s0, int buf) {
 #pragma unroll
     for (int i = 0; i < UN; ++i) {
       const int s = min(s0 + i, pl.S - 1);
       const int64_t sb = ((int64_t)b * pl.S + s) * pl.tiles + tile;
-      load_block_g(hend + sb * TILE_FLOATS, w.tid, he[buf][i]);
-      sd[buf][i] = w.act ? ldg_ch(segd + ((int64_t)b * pl.S + s) * pl.P + w.pa) : ch_zero();
+      he[buf][i] = __ldg(hend + sb * (TILE_FLOATS / 2) + in_blk);
+      sd[buf][i] = w.act ? __ldg(segd + ((int64_t)b * pl.S + s) * pl.P + w.pa + ch) : 0.f;
     }
   };
+  u64 hs = 0ull;
   auto apply = [&](int s0, int buf) {
 #pragma unroll
     for (int i = 0; i < UN; ++i) {
       const int s = s0 + i;
       if (s < pl.S) {
         const int64_t sb = ((int64_t)b * pl.S + s) * pl.tiles + tile;
-        store_block(hstart + sb * TILE_FLOATS, w.tid, hs);
-        u64 d2[NCH];
-#pragma unroll
-        for (int c = 0; c < NCH; ++c) d2[c] = pk(sd[buf][i].v[c], sd[buf][i].v[c]);
-#pragma unroll
-        for (int u = 0; u < NU; ++u) hs[u] = fma2(ex2_2(mul2(d2[u / 4], A2[u])), hs[u], he[buf][i][u]);
+        hstart[sb * (TILE_FLOATS / 2) + in_blk] = hs;
+        hs = fma2(ex2_2(mul2(pk(sd[buf][i], sd[buf][i]), A2u)), hs, he[buf][i]);
       }
     }
   };
@@ -1179,7 +1181,7 @@ int launch_prepass(const Plan& pl, const ScanPtrs& sp, bool with_mu, cudaStream_
 }
 
 int launch_fixup(const Plan& pl, const ScanPtrs& sp, bool with_mu, cudaStream_t st) {
-  fixup_h_kernel<<<dim3(pl.tiles, pl.B), NTHR, 0, st>>>(pl, sp.A_log, sp.ws);
+  fixup_h_kernel<<<dim3(pl.tiles, pl.B, NU), NTHR, 0, st>>>(pl, sp.A_log, sp.ws);
   count_launch();
   if (with_mu) {
     fixup_mu_kernel<<<dim3(pl.tiles, pl.full ? 1 : pl.S, pl.B), NTHR, 0, st>>>(pl, sp.A_log, sp.ws);
