@@ -293,7 +293,7 @@ __device__ __forceinline__ void zero_rows(uint8_t* tile, int row_bytes, int nt, 
 }
 
 template <typename IO, int MODE, bool SC>
-__global__ void __launch_bounds__(NTHR) ascend_kernel(const __grid_constant__ CUtensorMap tmX,
+__global__ void __launch_bounds__(NTHR, 4) ascend_kernel(const __grid_constant__ CUtensorMap tmX,
                                                     const __grid_constant__ CUtensorMap tmD,
                                                     const __grid_constant__ CUtensorMap tmG, Plan pl,
                                                     const float* __restrict__ A_log, char* __restrict__ ws,
@@ -333,7 +333,7 @@ __global__ void __launch_bounds__(NTHR) ascend_kernel(const __grid_constant__ CU
   if (w.tid == 0)
     for (int c = 0; c < NSTAGE && c < nchunk; ++c) issue(c);
 
-  u64 A2[NU], h[NU], Pr[NU], acc[NU], snap[NU];
+  u64 A2[NU], h[NU], Pr[NU], acc[NU];
   load_A2(A_log, w, A2, pl.scalar);
   const int64_t sb = ((int64_t)b * pl.S + s) * pl.tiles + tile;
   if (MODE == PRE_Y) {
@@ -343,10 +343,11 @@ __global__ void __launch_bounds__(NTHR) ascend_kernel(const __grid_constant__ CU
     for (int u = 0; u < NU; ++u) h[u] = 0ull;
   }
 #pragma unroll
-  for (int u = 0; u < NU; ++u) { Pr[u] = pk(1.f, 1.f); acc[u] = 0ull; snap[u] = 0ull; }
-  float cum[NCH], partd[NCH];
+  for (int u = 0; u < NU; ++u) { Pr[u] = pk(1.f, 1.f); acc[u] = 0ull; }
+  bool snapped = false;   // the r-token snapshot of acc and of the Delta sum goes straight to global memory when it is taken
+  float cum[NCH];
 #pragma unroll
-  for (int c = 0; c < NCH; ++c) { cum[c] = 0.f; partd[c] = 0.f; }
+  for (int c = 0; c < NCH; ++c) cum[c] = 0.f;
 
   for (int c = 0; c < nchunk; ++c) {
     const int st = c % NSTAGE;
@@ -424,10 +425,10 @@ __global__ void __launch_bounds__(NTHR) ascend_kernel(const __grid_constant__ CU
         for (int j = 0; j < CK; ++j) {
           token(j);
           if (j == jr) {
-#pragma unroll
-            for (int c = 0; c < NCH; ++c) partd[c] = cum[c];
-#pragma unroll
-            for (int u = 0; u < NU; ++u) snap[u] = acc[u];
+            store_block(reinterpret_cast<float*>(ws + pl.off_mupart) + sb * TILE_FLOATS, w.tid, acc);
+            if (w.half == 0 && w.act)
+              stg_ch(reinterpret_cast<float*>(ws + pl.off_partd) + ((int64_t)b * pl.S + s) * P + w.pa, cum);
+            snapped = true;
           }
         }
       } else {
@@ -443,21 +444,24 @@ __global__ void __launch_bounds__(NTHR) ascend_kernel(const __grid_constant__ CU
     if (w.tid == 0 && c + NSTAGE < nchunk) issue(c + NSTAGE);
   }
   if (MODE == PRE_Y) return;
-  if (MU && (t1 - t0) < pl.r) {   // ragged last segment shorter than r tokens: the snapshot is the whole segment
-#pragma unroll
-    for (int c = 0; c < NCH; ++c) partd[c] = cum[c];
-#pragma unroll
-    for (int u = 0; u < NU; ++u) snap[u] = acc[u];
-  }
   store_block(reinterpret_cast<float*>(ws + pl.off_hend) + sb * TILE_FLOATS, w.tid, h);
   const int64_t sp = ((int64_t)b * pl.S + s) * P + w.pa;
-  if (w.half == 0 && w.act) {
-    stg_ch(reinterpret_cast<float*>(ws + pl.off_segd) + sp, cum);
-    if (MU) stg_ch(reinterpret_cast<float*>(ws + pl.off_partd) + sp, partd);
-  }
+  if (w.half == 0 && w.act) stg_ch(reinterpret_cast<float*>(ws + pl.off_segd) + sp, cum);
   if (MU) {
     store_block(reinterpret_cast<float*>(ws + pl.off_muloc) + sb * TILE_FLOATS, w.tid, acc);
-    store_block(reinterpret_cast<float*>(ws + pl.off_mupart) + sb * TILE_FLOATS, w.tid, snap);
+    if (!snapped) {
+      // no r-th token in this segment: r = 0 (empty snapshot), or a ragged last segment shorter than r tokens (the
+      // snapshot is the whole segment)
+      const bool whole = (t1 - t0) < pl.r;
+      if (!whole) {
+#pragma unroll
+        for (int u = 0; u < NU; ++u) acc[u] = 0ull;
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) cum[c] = 0.f;
+      }
+      store_block(reinterpret_cast<float*>(ws + pl.off_mupart) + sb * TILE_FLOATS, w.tid, acc);
+      if (w.half == 0 && w.act) stg_ch(reinterpret_cast<float*>(ws + pl.off_partd) + sp, cum);
+    }
   }
 }
 
