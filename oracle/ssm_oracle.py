@@ -353,30 +353,38 @@ def rmsnorm_vjp(y, d, eps=RMS_EPS):
     return (d - yh * np.mean(d * yh, axis=-1, keepdims=True)) / r
 
 
-def stack_forward(thetas, y0):
-    """Section 3.2 / Alg. 1 lines 5-7 on one sequence: y_k = y_{k-1} + SSM_k(Norm(y_{k-1}))."""
+def stack_forward(thetas, y0, store=None):
+    """Section 3.2 / Alg. 1 lines 5-7 on one sequence: y_k = y_{k-1} + SSM_k(Norm(y_{k-1})).
+
+    `store`, if given, models the storage format of the activations: it is applied to every tensor
+    the stack keeps or hands from one layer to the next (the normalised input, the layer output,
+    the residual sum).  The default keeps everything in float64.  It changes no formula."""
+    keep = (lambda a: a) if store is None else store
     ys = [y0]
     yhats = []
     for th in thetas:
-        yhats.append(rmsnorm(ys[-1]))
-        ys.append(ys[-1] + ssm_forward(th, yhats[-1]))
+        yhats.append(keep(rmsnorm(ys[-1])))
+        ys.append(keep(ys[-1] + keep(ssm_forward(th, yhats[-1]))))
     return ys, yhats
 
 
-def stack_grad(thetas, y0, g, tbar, mode="chained", tier="direct"):
+def stack_grad(thetas, y0, g, tbar, mode="chained", tier="direct", store=None):
     """Gradients of every layer of the residual stack from one upstream g = dL/dy_K.
 
     mode "paper": Proposition 3 as printed - every layer receives g itself and its input
     Norm(y_{k-1}) is a constant.  mode "chained": true backpropagation through the stack,
-    G_K = g, G_{k-1} = G_k + RMSNormVJP(y_{k-1}, dx_k), layer k driven by G_k."""
-    ys, yhats = stack_forward(thetas, y0)
+    G_K = g, G_{k-1} = G_k + RMSNormVJP(y_{k-1}, dx_k), layer k driven by G_k.
+    `store` as in `stack_forward`; in the backward it is applied to the input gradient dx_k a layer
+    hands down and to the running upstream gradient G_k."""
+    keep = (lambda a: a) if store is None else store
+    ys, yhats = stack_forward(thetas, y0, store)
     K = len(thetas)
     grads = [None] * K
     G = g
     for k in range(K - 1, -1, -1):
         grads[k] = adjoint_grad(thetas[k], yhats[k], G if mode == "chained" else g, tbar, tier=tier)
         if mode == "chained":
-            G = G + rmsnorm_vjp(ys[k], grads[k]["dx"])
+            G = keep(G + rmsnorm_vjp(ys[k], keep(grads[k]["dx"])))
     return grads, (G if mode == "chained" else None)
 
 
