@@ -106,10 +106,24 @@ def oracle_sample_tokens_per_s(w, sample_T, verbose=False):
     theta = {k: synth.to_f64(v) for k, v in synth.layer_params(ws, 0, "cpu").items()}
     x, dy = synth.activations(ws, "cpu")
     x, dy = synth.to_f64(x), synth.to_f64(dy)
+    c0 = time.process_time()
     t0 = time.perf_counter()
     O.batched(O.adjoint_grad, theta, x, dy, ws.tbar, tier="block")
     dt = time.perf_counter() - t0
-    return sample_T / dt, dt, torch.get_num_threads()
+    cpu = time.process_time() - c0
+    return sample_T / dt, dt, cpu
+
+
+def cpu_baseline_record(w, sample_T, tps, dt, cpu):
+    """What the oracle run really used: the scans are single-threaded numpy loops over time, only the dense products
+    (projections, weight and input gradients) run on the BLAS thread pool; `cores` is CPU time / wall time."""
+    host = len(os.sched_getaffinity(0))
+    return {"value": tps, "unit": UNIT, "cores": max(1, round(cpu / dt)), "kind": "oracle",
+            "host_cores": host, "cpu_seconds": round(cpu, 2), "wall_seconds": round(dt, 2),
+            "threads": f"1 for the scans (numpy loops over time) + a BLAS pool of up to {host} for the dense products",
+            "sample": f"batch element 0, first {sample_T} tokens of {w.name}, Tbar={min(w.tbar, sample_T)}, all "
+                      f"{w.d_model} channels ({dt:.1f} s); the whole workload ({w.batch} x {w.seqlen} tokens) would take "
+                      f"about {w.batch * w.seqlen / tps:.0f} s, beyond the 10-30 s this leg is allowed"}
 
 
 def run_reference(args):
@@ -121,18 +135,18 @@ def run_reference(args):
     sample_T = args.cpu_sample_tokens
     vals = []
     for i in range(args.warmup + args.steps):
-        tps, dt, threads = oracle_sample_tokens_per_s(w, sample_T)
+        tps, dt, cpu = oracle_sample_tokens_per_s(w, sample_T)
         if i >= args.warmup:
-            vals.append((tps, dt))
+            vals.append((tps, dt, cpu))
     tps = sum(v[0] for v in vals) / len(vals)
     ms = 1e3 * sum(v[1] for v in vals) / len(vals)
-    sample = f"batch element 0, first {sample_T} tokens of {w.name}, Tbar=min({w.tbar},{sample_T}), all {w.d_model} channels"
+    base = cpu_baseline_record(w, sample_T, tps, ms * 1e-3, sum(v[2] for v in vals) / len(vals))
     line = {"impl": "reference", "metric": METRIC, "value": tps, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": w.name, "batch": 1, "seq_len": sample_T, "d_model": w.d_model,
                        "d_state": w.d_state, "tbar": min(w.tbar, sample_T)},
-            "cpu_baseline": {"value": tps, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "cpu_baseline": base,
             "e2e": {"value": tps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -216,12 +230,13 @@ def main():
     ms = e0.elapsed_time(e1) / args.steps
     # ---- per-phase timing (library-side CUDA events on the launching stream) ---------------------
     B.as_set_timing(True)
-    phase = {k: 0.0 for k in B.PHASES}
-    for _ in range(args.steps):
+    samples = {k: [] for k in B.PHASES}
+    for _ in range(max(args.steps, 5)):
         step()
         for k, v in B.as_get_timing().items():
-            phase[k] += v / args.steps
+            samples[k].append(v)
     B.as_set_timing(False)
+    phase = {k: statistics.median(v) for k, v in samples.items()}   # median over the steps: one slow call moves nothing
     # ---- end to end: pinned host inputs -> device, gradients -> host, inside the timed region -----
     if args.no_e2e:
         ms_e2e, h2d, d2h = float("nan"), 0, 0
@@ -238,20 +253,20 @@ def main():
 
 
 def run_e2e(args, torch, x, dy, grads, step, barrier, e0, e1):
-    """End to end with host buffers: every step copies its inputs from pinned host memory to the device and its
-    parameter gradients back.  The input copies run on a second stream into one of two device buffer sets, so
-    step i+1's host->device transfer overlaps step i's kernels (PCIe, not the kernels, bounds this figure)."""
-    from paper_2501_00692_b200 import binding as B
+    """End to end with host buffers: every step copies its inputs from pinned host memory to the device and every
+    result (the five parameter gradients and dx) back.  The input copies run on a second stream into one of two
+    device buffer sets, so step i+1's host->device transfer overlaps step i's kernels, and the dx read-back runs on a
+    third stream from a device copy the next step does not overwrite (PCIe, not the kernels, bounds this figure)."""
     xh, dyh = x.cpu().pin_memory(), dy.cpu().pin_memory()
-    outh = {k: torch.empty_like(v, device="cpu").pin_memory() for k, v in grads.items() if k != "dx"}
+    outh = {k: torch.empty_like(v, device="cpu").pin_memory() for k, v in grads.items() if v is not None}
     h2d = xh.numel() * xh.element_size() * 2
     d2h = sum(v.numel() * v.element_size() for v in outh.values())
     bufs = [(x, dy), (torch.empty_like(x), torch.empty_like(dy))]
-    copy_stream = torch.cuda.Stream()
+    copy_stream, back_stream = torch.cuda.Stream(), torch.cuda.Stream()
     main = torch.cuda.current_stream()
     copied = [torch.cuda.Event() for _ in range(2)]
     consumed = [torch.cuda.Event() for _ in range(2)]
-    step_fn = step   # step(xbuf, dybuf)
+    produced, drained = torch.cuda.Event(), torch.cuda.Event()
 
     def run(n):
         for i in range(n):
@@ -262,10 +277,17 @@ def run_e2e(args, torch, x, dy, grads, step, barrier, e0, e1):
                 xb.copy_(xh, non_blocking=True); dyb.copy_(dyh, non_blocking=True)
                 copied[i % 2].record(copy_stream)
             main.wait_event(copied[i % 2])
-            step_fn(xb, dyb)
+            if i >= 1:
+                main.wait_event(drained)                         # the previous step's results have left the device buffers
+            step(xb, dyb)
             consumed[i % 2].record(main)
-            for k, v in outh.items():
-                v.copy_(grads[k], non_blocking=True)
+            produced.record(main)
+            with torch.cuda.stream(back_stream):
+                back_stream.wait_event(produced)
+                for k, v in outh.items():
+                    v.copy_(grads[k], non_blocking=True)
+                drained.record(back_stream)
+        main.wait_stream(back_stream)
 
     run(2); torch.cuda.synchronize()
     barrier(); torch.cuda.synchronize()
@@ -285,53 +307,78 @@ def l2_note(w, tokens):
     return f"inputs fit in L2 ({gb * 1e3:.0f} MB per step): parity workload, not a roofline measurement"
 
 
+# Per state-step (token, channel, state) work of the main adjoint kernel.
+# The method's own count: 1 ex2 (abar_i) + 1 more where the window-exit factor is live, and 12 FP32-pipe operations
+# (rebuild h: 3; mu: 2; dC, dB, s: 3; abar h mu and its two sums: 4).  What this build's kernel executes on top of that is
+# stated separately, so that redundancy shows instead of being credited.
+METHOD_EX2_PER_STATE_STEP = 1.0
+METHOD_FMA_PER_STATE_STEP = 12.0
+KERNEL_EX2_PER_STATE_STEP = {"forward rebuild of the chunk (abar)": 1.0, "backward walk (abar again)": 1.0,
+                             "chunk-start fix-up": 1.0 / 8}
+# measured pipe rates per clock per SM (profiles/pipe_rates_microbenchmark.md)
+MUFU_PER_CLK_SM = 16.0
+FMA_PER_CLK_SM = 128.0
+
+
 def report(args, B, w, world, rank, tokens, ms, ms_e2e, h2d, d2h, launches, phase, clocks):
     if rank == 0:
         peak, peak_src = measured_peaks()
         e = 2 if w.io == "bf16" else 4
-        # algorithmic bytes of the main adjoint kernel per token: read x, dy (2 P e) and Delta (4 P); write du, dx_dir (2 P e);
-        # read [B|C] and write [dB|dC] (2 x 2N fp32)
-        bytes_per_token = w.d_model * (2 * e + 4 + 2 * e) + 2 * (2 * w.d_state * 4)
+        P, N = w.d_model, w.d_state
+        # algorithmic bytes of the main adjoint kernel per token: read x, dy (2 P e), Delta (4 P), B_t, C_t (2 N e);
+        # write du, dx_dir (2 P e) and dB_t, dC_t (2 N fp32)
+        bytes_per_token = P * (4 * e + 4) + 2 * N * e + 2 * N * 4
         k_ms = phase["adjoint_main"]
         achieved = bytes_per_token * tokens / (k_ms * 1e-3) / 1e9 if k_ms > 0 else None
-        # MUFU issue bound of the same kernel: >= 2 ex2 per (token, channel, state) in the chunk walk + 1/8 for the
-        # checkpoint fix-up + 1/16 for the sigmoid; 16 ex2 per clock per SM (measured), at the sampled SM clock
         sm_mhz = (clocks or {}).get("sm_mhz") or 1965.0
-        ex2 = tokens * w.d_model * w.d_state * (2.0 + 1.0 / 8) + tokens * w.d_model
-        alu_peak = 16 * 148 * sm_mhz * 1e6
-        alu = {"kernel": "adjoint_main_kernel", "bound": "alu", "pipe": "MUFU.EX2", "achieved": ex2 / (k_ms * 1e-3) if k_ms > 0 else None,
-               "peak": alu_peak, "unit": "ex2/s", "frac": (ex2 / (k_ms * 1e-3) / alu_peak) if k_ms > 0 else None,
-               "peak_source": "16 ex2/clk/SM (measured) x 148 SMs x sampled SM clock", "sm_mhz": sm_mhz,
-               "ops_per_launch": ex2}
+        sms = B.as_sm_count()
+        steps = tokens * P * N
+        live = 1.0 if args.slow_decay else 0.0            # the window-exit factor is live under the slow-decay law only
+        ex2_method = steps * (METHOD_EX2_PER_STATE_STEP + live)
+        fma_method = steps * METHOD_FMA_PER_STATE_STEP
+        ex2_exec = steps * (sum(KERNEL_EX2_PER_STATE_STEP.values()) + live) + tokens * P      # + sigmoid per (token, channel)
+        mufu_peak = MUFU_PER_CLK_SM * sms * sm_mhz * 1e6
+        fma_peak = FMA_PER_CLK_SM * sms * sm_mhz * 1e6
+        sec = k_ms * 1e-3
+        alu = {"kernel": "adjoint_main_kernel", "bound": "alu", "sm_mhz": sm_mhz, "launch_ms": k_ms,
+               "peak_source": f"{MUFU_PER_CLK_SM:g} ex2 and {FMA_PER_CLK_SM:g} FP32 FMA lanes per clock per SM (measured, "
+                              f"profiles/pipe_rates_microbenchmark.md) x {sms} SMs x sampled SM clock",
+               "method_ops": {"ex2_per_state_step": METHOD_EX2_PER_STATE_STEP + live, "fma_per_state_step": METHOD_FMA_PER_STATE_STEP},
+               "mufu": {"achieved": ex2_method / sec, "peak": mufu_peak, "unit": "ex2/s", "frac": ex2_method / sec / mufu_peak},
+               "fma": {"achieved": fma_method / sec, "peak": fma_peak, "unit": "FP32 op/s", "frac": fma_method / sec / fma_peak},
+               "executed_ex2": {"per_state_step": KERNEL_EX2_PER_STATE_STEP, "per_launch": ex2_exec,
+                                "frac_of_mufu_peak": ex2_exec / sec / mufu_peak}} if k_ms > 0 else None
         traffic = None
         tpath = os.path.join(ROOT, "profiles", "traffic.json")
         if os.path.exists(tpath):
             traffic = json.load(open(tpath)).get(f"adjoint_main_kernel:{w.name}")
+        psum = sum(phase.values())
         line = {"metric": METRIC, "value": job_value(tokens, world, ms), "unit": UNIT, "n_gpus": world,
                 "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "scaling": "weak", "vs_baseline": None,
+                "dtype": "f32" if w.io == "f32" else "bf16 (fp32 accum)", "data": "synthetic",
                 "config": {"workload": w.name, "batch": w.batch, "seq_len": w.seqlen, "d_model": w.d_model,
                            "d_state": w.d_state, "tbar": w.tbar, "io": w.io, "layers": 1,
                            "parallelism": "replicas only" if world > 1 else "single GPU",
                            "l2": l2_note(w, tokens)},
                 "e2e": {"value": job_value(tokens, world, ms_e2e) if ms_e2e == ms_e2e else None, "unit": UNIT, "h2d_bytes_per_step": h2d,
-                        "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e if ms_e2e == ms_e2e else None},
+                        "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e if ms_e2e == ms_e2e else None,
+                        "results_copied_back": "dW_delta, db_delta, dW_B, dW_C, dA_log, dx"},
                 "gpu_launches": launches,
-                "phases_ms": phase,
-                # the binding roofline of the dominant kernel: MUFU.EX2 issue (the kernel is ALU/SFU-bound, DRAM ~13 % busy)
-                "roofline": dict(alu, traffic=traffic, launch_ms=k_ms),
-                # the metric's named roofline: algorithmic HBM bytes / kernel time against the measured copy bandwidth
-                "roofline_hbm": {"kernel": "adjoint_main_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
-                                 "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "traffic": traffic,
-                                 "peak_source": peak_src, "bytes_per_launch": bytes_per_token * tokens,
-                                 "launch_ms": k_ms},
+                "phases_ms": phase, "phases_sum_ms": psum, "phases_stat": "median over the steps",
+                "phases_consistent": abs(psum - ms) <= 0.05 * ms,
+                # the metric's named roofline: algorithmic HBM bytes of the dominant kernel / its launch time (library-side
+                # CUDA events on the launching stream) against the measured copy bandwidth
+                "roofline": {"kernel": "adjoint_main_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
+                             "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "traffic": traffic,
+                             "peak_source": peak_src, "bytes_per_token": bytes_per_token,
+                             "bytes_per_launch": bytes_per_token * tokens, "launch_ms": k_ms},
+                # what actually binds the kernel: MUFU / FP32 issue, on the method's own operation count
+                "roofline_alu": alu,
                 "clocks": clocks}
         if world == 1 and not args.no_cpu_baseline:
-            tps, dt, threads = oracle_sample_tokens_per_s(w, args.cpu_sample_tokens)
-            line["cpu_baseline"] = {"value": tps, "unit": UNIT, "cores": threads, "kind": "oracle",
-                                    "sample": f"batch element 0, first {args.cpu_sample_tokens} tokens of {w.name}, "
-                                              f"Tbar={min(w.tbar, args.cpu_sample_tokens)}, all {w.d_model} channels "
-                                              f"({dt:.1f} s)"}
+            tps, dt, cpu = oracle_sample_tokens_per_s(w, args.cpu_sample_tokens)
+            line["cpu_baseline"] = cpu_baseline_record(w, args.cpu_sample_tokens, tps, dt, cpu)
         print(json.dumps(line))
 
 

@@ -11,13 +11,25 @@
  * Conventions for every entry point
  *   - Every tensor pointer is a DEVICE pointer owned by the caller, contiguous, row-major (last index
  *     fastest) and 16-byte aligned.  Activations are [batch, seqlen, d_model]; "io dtype" is fp32 or
- *     bf16 as selected by as_shape_t.io.  The library never allocates, frees or keeps device memory.
+ *     bf16 as selected by as_shape_t.io.  The library never allocates or frees device memory, and keeps none
+ *     between calls, with one exception: the fixed scratch array of as_ssm_forward_static (see there).
  *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the legacy default
  *     stream).  No entry point synchronises except as_check_status.
  *   - `ws` is caller-provided scratch of at least the size reported by as_workspace_bytes; its
  *     contents on entry are ignored and on return are unspecified.
  *   - Return value: AS_OK (0) or a negative AS_ERR_* code.  Nothing is launched when an argument
  *     check fails.  No exceptions, no aborts, no printing.
+ *   - Threads: the entry points keep no shared mutable state, so several host threads may call them at once
+ *     (each call with its own `ws`), except for the phase-timing diagnostic (one thread, one stream) and the
+ *     shared array of as_ssm_forward_static.  The library uses the CUDA runtime API, i.e. each device's primary context.
+ *   - Size limits (AS_ERR_LIMIT): batch * seqlen + seqlen + 16 < 2^31 (token rows are 32-bit TMA coordinates) and
+ *     seqlen <= 65535 * 2048 (time segments fill one grid dimension).
+ *   - Device-side waits: every wait on staged data (mbarrier waits on TMA / bulk copies and on tensor-core commits)
+ *     is bounded and ends in AS_ERR_TIMEOUT.  The one wait that has no software bound is the hardware allocation of
+ *     tensor memory (tcgen05.alloc) at the start of the contraction and adjoint kernels: it blocks until enough of
+ *     the SM's 512 columns are free, which happens when CTAs that hold them finish; a kernel of this library frees
+ *     its columns on every exit path and never waits for another CTA while holding them, so the allocation of a
+ *     later CTA always completes.
  *   - Results are deterministic up to floating-point summation order (fp32 atomics are used for the
  *     sums over channels, segments and the batch).
  */
@@ -31,7 +43,7 @@
 extern "C" {
 #endif
 
-#define AS_VERSION 101
+#define AS_VERSION 102
 
 typedef enum { AS_F32 = 0, AS_BF16 = 1 } as_dtype_t;
 
@@ -93,7 +105,8 @@ const char *as_strerror(int code);
 int as_workspace_bytes(const as_shape_t *shape, int64_t tbar, size_t *fwd_bytes, size_t *grad_bytes);
 
 /* Synchronises `stream` and returns the status word the kernels keep at the start of `ws`
- * (AS_OK, or AS_ERR_TIMEOUT if a bounded device-side wait ran out). */
+ * (AS_OK, or AS_ERR_TIMEOUT if a bounded device-side wait ran out).  ws == NULL selects the built-in scratch
+ * array of as_ssm_forward_static on the current device. */
 int as_check_status(const void *ws, void *stream);
 
 /* SSM(X) = Y (Section 3.1, steps 1-5; Alg. 1 line 5 for one layer).
@@ -132,6 +145,8 @@ int as_full_bptt_grad(const as_shape_t *shape, const as_params_t *params, const 
  *     device current): make it during set-up, before any stream capture;
  *   - all calls on a device share the array and it keeps the previous call's contents (what must start at zero is
  *     cleared by the call); calls whose kernels may overlap on the GPU race on it - order them on one stream;
+ *   - the status word of the call's kernels sits at the head of the array: read it with as_check_status(NULL, stream);
+ *   - the array belongs to the device's primary context (the one the CUDA runtime API uses);
  *   - neither this call nor anything it launches calls cudaMalloc, cudaFree or another allocating routine.
  * x, y: [Bsz,T,P] io dtype device buffers supplied by the caller, as for as_ssm_forward. */
 #define AS_STATIC_SCRATCH_BYTES (32u << 20)
@@ -160,10 +175,14 @@ int as_wait_selftest(void *ws, size_t ws_bytes, uint32_t poll_limit, void *strea
 
 /* host-side bookkeeping only; no effect on results */
 
+/* Number of SMs of the current device as the library sees it (grids are sized in multiples of it). */
+int as_sm_count(void);
+
 /* Number of kernels this library has launched in this process since the last reset; reset != 0 zeroes it. */
 int64_t as_launch_count(int reset);
 
-/* Phase timing of as_adjoint_grad.  as_set_timing(1) makes every later as_adjoint_grad call record CUDA
+/* Phase timing of as_adjoint_grad (process-wide state, not thread-safe: use it from one host thread driving one
+ * stream).  as_set_timing(1) makes every later as_adjoint_grad call record CUDA
  * events on its stream between its phases (this creates the events once; timing mode is opt-in and is the one
  * place where the library creates CUDA objects).  as_get_timing synchronises on the last event of the most
  * recent call and writes elapsed milliseconds into ms[0..AS_NUM_PHASES): projections (S1, incl. zeroing),

@@ -23,7 +23,7 @@ AS_ERR_WORKSPACE, AS_ERR_ALIGN, AS_ERR_CUDA, AS_ERR_TIMEOUT, AS_ERR_LIMIT = -5, 
 
 EXPORTS = ("as_version", "as_strerror", "as_workspace_bytes", "as_check_status", "as_ssm_forward",
            "as_adjoint_grad", "as_full_bptt_grad", "as_rmsnorm_fwd", "as_residual_add", "as_rmsnorm_bwd_add",
-           "as_launch_count", "as_set_timing", "as_get_timing", "as_ssm_forward_static", "as_wait_selftest")
+           "as_launch_count", "as_set_timing", "as_get_timing", "as_ssm_forward_static", "as_wait_selftest", "as_sm_count")
 AS_STATIC_SCRATCH_BYTES = 32 << 20
 AS_NUM_PHASES = 6
 PHASES = ("projections", "prepass", "fixup", "adjoint_main", "weight_grads", "input_grad")
@@ -157,8 +157,13 @@ def as_workspace_bytes(shape: as_shape_t, tbar: int):
     return fwd.value, grad.value
 
 
-def as_check_status(ws: torch.Tensor, stream=None) -> int:
+def as_check_status(ws, stream=None) -> int:
+    """Status word of the kernels that used `ws`; ws=None reads the built-in scratch of as_ssm_forward_static."""
     return lib().as_check_status(_ptr(ws), _stream(stream))
+
+
+def as_sm_count() -> int:
+    return int(lib().as_sm_count())
 
 
 def as_ssm_forward(shape, theta, x, y, ws, stream=None):

@@ -11,6 +11,8 @@ std::atomic<int64_t> g_launches{0};
 
 namespace {
 
+// Phase timing is a diagnostic with process-wide state: one set of events, no locking.  It is meant for one host
+// thread driving one stream (as the header says); everything else in the library is free of shared mutable state.
 bool g_timing = false;
 bool g_timing_valid = false;
 cudaEvent_t g_ev[AS_NUM_PHASES + 1];
@@ -29,6 +31,9 @@ int check_shape(const as_shape_t* sh) {
   if (sh->io != AS_F32 && sh->io != AS_BF16) return AS_ERR_DTYPE;
   if (sh->d_model % 8 != 0) return AS_ERR_ALIGN;
   if (sh->batch > 65535) return AS_ERR_SHAPE;
+  // token rows are addressed with 32-bit TMA coordinates (row + window lookahead + one chunk), and the time
+  // segments (at most 2048 tokens each) fill gridDim.y
+  if ((int64_t)sh->batch * sh->seqlen + sh->seqlen + 2 * CK >= ((int64_t)1 << 31)) return AS_ERR_LIMIT;
   return AS_OK;
 }
 
@@ -71,7 +76,7 @@ int projections(const Plan& pl, const as_params_t* pr, const void* x, char* ws, 
 }
 
 int pick_splitk(int64_t tiles, int64_t K) {
-  int64_t s = (148 * 4 + tiles - 1) / tiles;
+  int64_t s = ((int64_t)sm_count() * 4 + tiles - 1) / tiles;
   const int64_t maxs = (K + 255) / 256;
   if (s > maxs) s = maxs;
   if (s < 1) s = 1;
@@ -183,14 +188,20 @@ int as_workspace_bytes(const as_shape_t* shape, int64_t tbar, size_t* fwd_bytes,
   if (e) return e;
   if (tbar < 1) return AS_ERR_TBAR;
   Plan pl;
-  make_plan(shape, tbar, &pl);
+  e = make_plan(shape, tbar, &pl);
+  if (e) return e;
   if (fwd_bytes) *fwd_bytes = pl.total_fwd;
   if (grad_bytes) *grad_bytes = pl.total_grad;
   return AS_OK;
 }
 
 int as_check_status(const void* ws, void* stream) {
-  if (!ws) return AS_ERR_NULL;
+  if (!ws) {   // the built-in scratch array of as_ssm_forward_static on the current device
+    void* p = nullptr;
+    const int e = static_scratch_address(&p);
+    if (e) return e;
+    ws = p;
+  }
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   int word = 0;
   if (cudaMemcpyAsync(&word, ws, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return AS_ERR_CUDA;
@@ -207,7 +218,8 @@ int as_ssm_forward(const as_shape_t* shape, const as_params_t* params, const voi
   if (!x || !y || !ws) return AS_ERR_NULL;
   if (!aligned16(x) || !aligned16(y) || !aligned16(ws)) return AS_ERR_ALIGN;
   Plan pl;
-  make_plan(shape, shape->seqlen, &pl);
+  e = make_plan(shape, shape->seqlen, &pl);
+  if (e) return e;
   if (ws_bytes < pl.total_fwd) return AS_ERR_WORKSPACE;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   char* w = reinterpret_cast<char*>(ws);
@@ -227,7 +239,8 @@ int as_adjoint_grad(const as_shape_t* shape, const as_params_t* params, const vo
   if (e) return e;
   if (tbar < 1) return AS_ERR_TBAR;
   Plan pl;
-  make_plan(shape, tbar, &pl);
+  e = make_plan(shape, tbar, &pl);
+  if (e) return e;
   if (ws_bytes < pl.total_grad) return AS_ERR_WORKSPACE;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   char* w = reinterpret_cast<char*>(ws);
@@ -254,7 +267,8 @@ int as_full_bptt_grad(const as_shape_t* shape, const as_params_t* params, const 
   int e = check_grad_args(shape, params, x, dy, out, ws);
   if (e) return e;
   Plan pl;
-  make_plan(shape, shape->seqlen, &pl);
+  e = make_plan(shape, shape->seqlen, &pl);
+  if (e) return e;
   if (ws_bytes < pl.total_grad) return AS_ERR_WORKSPACE;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   char* w = reinterpret_cast<char*>(ws);
@@ -308,6 +322,8 @@ int64_t as_launch_count(int reset) {
   if (reset) as::g_launches.store(0);
   return v;
 }
+
+int as_sm_count(void) { return sm_count(); }
 
 int as_set_timing(int enable) {
   static bool created = false;

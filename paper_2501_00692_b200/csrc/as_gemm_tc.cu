@@ -473,7 +473,8 @@ int launch_tc(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap 
   static bool done[AS_MAX_DEVICES] = {};
   if (ensure_dynamic_smem(kern, Cfg<BN>::SMEM_DYN, done)) return 1;
   const int64_t ntiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN) * a.splitk;
-  const unsigned grid = (unsigned)(ntiles < 148 ? ntiles : 148);   // one persistent CTA per SM
+  const int sms = sm_count();
+  const unsigned grid = (unsigned)(ntiles < sms ? ntiles : sms);   // one persistent CTA per SM
   kern<<<grid, NTHREADS, Cfg<BN>::SMEM_DYN, st>>>(tmA, tmB, tmO[0], tmO[1], tmO[2], a);
   count_launch();
   return (int)cudaGetLastError();
@@ -523,7 +524,7 @@ int tc_weight_grads(const Plan& pl, const void* x, const as_grads_t* out, char* 
   TcArgs a{};
   a.M = NW; a.N = P; a.kblocks = (int)((M + BK - 1) / BK); a.P = P;
   const int tiles = ((NW + BM - 1) / BM) * ((P + TBN - 1) / TBN);
-  int sk = (148 * 2) / tiles;   // about two tiles per persistent CTA
+  int sk = (sm_count() * 2) / tiles;   // about two tiles per persistent CTA
   if (sk > a.kblocks) sk = a.kblocks;
   if (sk < 1) sk = 1;
   const int kper = (a.kblocks + sk - 1) / sk;

@@ -19,7 +19,7 @@ inline void count_launch(int n = 1) { g_launches.fetch_add(n); }
 // instantiation, whether the limit has been raised.  `done` is a static array of the launcher, one flag per device.
 constexpr int AS_MAX_DEVICES = 64;
 template <typename K>
-inline int ensure_dynamic_smem(K kern, int bytes, bool (&done)[AS_MAX_DEVICES]) {
+inline int ensure_dynamic_smem(K kern, int bytes, bool (&done)[AS_MAX_DEVICES]) {   // idempotent: a race between host threads only repeats the call
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= AS_MAX_DEVICES) return 1;
   if (!done[dev]) {
@@ -27,6 +27,20 @@ inline int ensure_dynamic_smem(K kern, int bytes, bool (&done)[AS_MAX_DEVICES]) 
     done[dev] = true;
   }
   return 0;
+}
+
+// Number of SMs of the current device (grids are sized in multiples of it); queried once per device.  The cache is
+// a plain array of atomics: concurrent first calls from several host threads at worst query twice.
+inline int sm_count() {
+  static std::atomic<int> cached[AS_MAX_DEVICES] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= AS_MAX_DEVICES) return 148;
+  int n = cached[dev].load(std::memory_order_relaxed);
+  if (n <= 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached[dev].store(n, std::memory_order_relaxed);
+  }
+  return n;
 }
 
 constexpr int NS = 16;        // d_state handled by the scan kernels
@@ -121,6 +135,9 @@ int tc_weight_grads(const Plan& pl, const void* x, const as_grads_t* out, char* 
 int tc_input_grad(const Plan& pl, void* dx, char* ws, cudaStream_t st);
 
 int launch_bptt(const Plan& pl, const ScanPtrs& sp, float* dA_log, float* db_delta, cudaStream_t st);
+
+// device address of the library's built-in scratch array on the current device (as_noalloc.cu); AS_OK or an error code
+int static_scratch_address(void** out);
 
 int launch_rmsnorm_fwd(const as_shape_t* sh, const void* y, void* yhat, float eps, cudaStream_t st);
 int launch_residual_add(const as_shape_t* sh, const void* a, const void* b, void* out, cudaStream_t st);

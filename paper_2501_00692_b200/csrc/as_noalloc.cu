@@ -27,7 +27,10 @@ namespace {
 static __device__ __align__(256) unsigned char g_static_scratch[AS_STATIC_SCRATCH_BYTES];
 
 constexpr int kMaxDevices = 64;
-void* g_scratch_addr[kMaxDevices] = {};   // device address of g_static_scratch, per device ordinal
+// Device address of g_static_scratch per device ordinal, in the device's primary context (the context the CUDA runtime
+// API uses; a caller that makes its own driver-API contexts current is not supported by this entry point).  Atomic so
+// that host threads may make their first calls concurrently: both would store the same address.
+std::atomic<void*> g_scratch_addr[kMaxDevices] = {};
 
 // The name g_static_scratch is, in host code, only a handle for the runtime: it is not a device address and
 // must never be passed to a kernel.  The address a kernel can use comes from cudaGetSymbolAddress, queried
@@ -36,16 +39,20 @@ int scratch_for_current_device(void** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) return AS_ERR_CUDA;
   if (dev < 0 || dev >= kMaxDevices) return AS_ERR_LIMIT;
-  if (!g_scratch_addr[dev]) {
-    void* p = nullptr;
+  void* p = g_scratch_addr[dev].load(std::memory_order_acquire);
+  if (!p) {
     if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return AS_ERR_CUDA;
-    g_scratch_addr[dev] = p;
+    g_scratch_addr[dev].store(p, std::memory_order_release);
   }
-  *out = g_scratch_addr[dev];
+  *out = p;
   return AS_OK;
 }
 
 }  // namespace
+
+// The status word of as_ssm_forward_static lives at the head of the static array: as_check_status(NULL, stream)
+// reads it through this.
+int as::static_scratch_address(void** out) { return scratch_for_current_device(out); }
 
 extern "C" int as_ssm_forward_static(const as_shape_t* shape, const as_params_t* params, const void* x, void* y,
                                      void* stream) {

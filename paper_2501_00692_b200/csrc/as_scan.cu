@@ -35,7 +35,7 @@ int make_plan(const as_shape_t* sh, int64_t tbar, Plan* pl) {
   p.bw = p.P < CH ? p.P : CH;
   const int64_t ctas = (int64_t)p.tiles * p.B;
   // two full waves of the main kernel's resident CTAs (148 SMs x CTAs per SM), never more than that
-  const int64_t slots = 148 * 3;
+  const int64_t slots = (int64_t)sm_count() * 3;
   int64_t s_target = (2 * slots) / ctas;
   if (s_target < 1) s_target = 1;
   int64_t L = (p.T + s_target - 1) / s_target;
@@ -76,7 +76,7 @@ int make_plan(const as_shape_t* sh, int64_t tbar, Plan* pl) {
   p.off_bptt_ckpt = take((size_t)p.B * ((p.T + 63) / 64) * p.P * NS * 4);
   p.total_grad = o;
   *pl = p;
-  return AS_OK;
+  return p.S > 65535 ? AS_ERR_LIMIT : AS_OK;   // segments fill gridDim.y
 }
 
 namespace {
@@ -438,7 +438,13 @@ __global__ void __launch_bounds__(NTHR, 4) ascend_kernel(const __grid_constant__
     }
     const int bad = __syncthreads_or(ok ? 0 : 1);
     if (bad) {
-      if (w.tid == 0) atomicExch(status, AS_ERR_TIMEOUT);
+      if (w.tid == 0) {
+        // copies issued for this and the following chunks still target this CTA's shared memory: give each one more
+        // bounded wait before the CTA (and its shared memory) goes away
+        for (int c2 = c; c2 < nchunk && c2 < c + NSTAGE; ++c2) mbar_wait(&full_bar[c2 % NSTAGE], (c2 / NSTAGE) & 1);
+        atomicExch(status, AS_ERR_TIMEOUT);
+      }
+      __syncthreads();
       return;
     }
     if (w.tid == 0 && c + NSTAGE < nchunk) issue(c + NSTAGE);
@@ -793,6 +799,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   }
   float dbacc = 0.f;
   bool failed = false;
+  int fail_i = 0, ckp_issued = 0;   // thread 0: where the walk stopped, last checkpoint copy issued
 
   for (int i = 0; i < nchunk; ++i) {
     const int st = i % NSTAGE_MAIN;
@@ -885,7 +892,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
       }
       if (w.tid == 0 && i + 1 < nchunk) {
         // every thread has copied the checkpoint into registers long ago: fetch the next chunk's
-        if (mbar_wait(&ckp_free, i & 1)) issue_ckp(i + 1);
+        if (mbar_wait(&ckp_free, i & 1)) { issue_ckp(i + 1); ckp_issued = i + 1; }
         else tfail = true;
       }
       // output rows of this chunk, walked from its last token down
@@ -1028,7 +1035,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     }
     (void)swl;
     const int bad = __syncthreads_or((ok && !tfail) ? 0 : 1);
-    if (bad) { failed = true; break; }
+    if (bad) { failed = true; fail_i = i; break; }
     if (w.tid == 0 && i + NSTAGE_MAIN < nchunk) issue(i + NSTAGE_MAIN);
     for (int e = w.tid; e < CK * NBC; e += NTHR) {
       const int j = e / NBC, q = e % NBC;
@@ -1037,7 +1044,13 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     }
   }
   if (failed) {
-    if (w.tid == 0) atomicExch(status, AS_ERR_TIMEOUT);
+    if (w.tid == 0) {
+      // copies already issued still target this CTA's shared memory: one more bounded wait for each before leaving
+      for (int i2 = fail_i; i2 < nchunk && i2 < fail_i + NSTAGE_MAIN; ++i2)
+        mbar_wait(&full_bar[i2 % NSTAGE_MAIN], (i2 / NSTAGE_MAIN) & 1);
+      mbar_wait(&ckp_bar, ckp_issued & 1);
+      atomicExch(status, AS_ERR_TIMEOUT);
+    }
   } else {
     if (w.act && !pl.scalar) {
 #pragma unroll

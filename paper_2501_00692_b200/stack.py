@@ -76,9 +76,9 @@ class Stack:
         grads = [None] * self.K
         for k in range(self.K - 1, -1, -1):
             st, ws, yhat = lanes[k % len(lanes)]
+            gk = B.alloc_grads(self.shape, g.device, with_dx=False)   # allocated on the main stream, which joins below
             with torch.cuda.stream(st):
                 B.as_rmsnorm_fwd(self.shape, self.ys[k], yhat, self.eps)
-                gk = B.alloc_grads(self.shape, g.device, with_dx=False)
                 B.as_adjoint_grad(self.shape, self.thetas[k], yhat, g, self.tbar, gk, ws)
             grads[k] = gk
         for st, _, _ in self.extra:

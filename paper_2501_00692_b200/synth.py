@@ -112,13 +112,16 @@ def custom_workload(name, config, batch, seqlen, d_model, d_state=16, layers=1, 
                     seqlen if tbar is None else tbar, io)
 
 
-def layer_params(w: Workload, layer: int = 0, device="cpu", slow_decay: bool = False) -> dict:
-    """Parameters of layer `layer`: W_* in the I/O dtype, b_delta and A_log in fp32."""
+def layer_params(w: Workload, layer: int = 0, device="cpu", slow_decay: bool = False, b_delta_range=None) -> dict:
+    """Parameters of layer `layer`: W_* in the I/O dtype, b_delta and A_log in fp32.
+    `b_delta_range` (lo, hi) overrides the law of b_delta, e.g. (-1, 1) for a fast-decay corner (abar << 1)."""
     base = 1000 * w.config + 17 * layer
     P, N = w.d_model, w.d_state
     dt = w.torch_dtype
     std = 1.0 / math.sqrt(P)
     lo, hi = (-9.0, -7.0) if slow_decay else (-4.0, -2.0)
+    if b_delta_range is not None:
+        lo, hi = float(b_delta_range[0]), float(b_delta_range[1])
     return {
         "W_delta": _fill("normal", base + TID_W_DELTA, (P, P), device, dt, scale=std),
         "b_delta": _fill("uniform", base + TID_B_DELTA, (P,), device, torch.float32, lo=lo, hi=hi),

@@ -30,6 +30,11 @@ def _block(args):
     return out
 
 
+def _fwd_block(args):
+    delta, xs, Bm, Cm, A = args
+    return O.scan_forward(delta, xs, Bm, Cm, A)[0]
+
+
 _POOL = None
 
 
@@ -41,6 +46,40 @@ def pool(workers=None):
     return _POOL
 
 
+def host_memory_gb():
+    """Memory this process may still use: the smaller of the host's available memory and the cgroup's headroom."""
+    avail = 1e9
+    try:
+        for line in open("/proc/meminfo"):
+            if line.startswith("MemAvailable:"):
+                avail = int(line.split()[1]) / 2 ** 20
+    except OSError:
+        pass
+    try:
+        lim = open("/sys/fs/cgroup/memory.max").read().strip()
+        if lim != "max":
+            avail = min(avail, (int(lim) - int(open("/sys/fs/cgroup/memory.current").read())) / 2 ** 30)
+    except (OSError, ValueError):
+        pass
+    return avail
+
+
+def map_bounded(fn, jobs, gb_per_job):
+    """pool().map in rounds small enough that the jobs running at once fit in half of the memory available."""
+    p = pool()
+    n = int(max(1, min(p._processes, 0.5 * host_memory_gb() // max(gb_per_job, 1e-3))))
+    out = []
+    for i in range(0, len(jobs), n):
+        part = jobs[i:i + n]
+        out += p.map(fn, part, chunksize=1) if len(part) > 1 else [fn(part[0])]
+    return out
+
+
+def _scan_gb(T, channels, states):
+    """Rough peak of one _block job: about seven [T, channels, states] fp64 arrays."""
+    return 7 * T * channels * states * 8 / 2 ** 30
+
+
 def channel_scans(theta, x, g, tbar, tier="block", channel_block=32, channels=None, want=()):
     """Per-channel results of one sequence for `channels` (default: all): y, du, dx_dir, dA_log per channel, and the
     channel sums dB, dC over the channels given.  Returns a dict of arrays indexed like `channels`."""
@@ -50,7 +89,7 @@ def channel_scans(theta, x, g, tbar, tier="block", channel_block=32, channels=No
     for p0 in range(0, len(sel), channel_block):
         s = sel[p0:p0 + channel_block]
         jobs.append((delta[:, s], x[:, s], u[:, s], g[:, s], Bm, Cm, A[s], tbar, tier, tuple(want)))
-    res = pool().map(_block, jobs) if len(jobs) > 1 else [_block(j) for j in jobs]
+    res = map_bounded(_block, jobs, _scan_gb(x.shape[0], channel_block, A.shape[1]))
     out = {k: np.concatenate([r[k] for r in res], axis=1) for k in ("y", "du", "dx_dir")}
     out["dA_log"] = np.concatenate([r["dA_log"] for r in res], axis=0)
     out["dB"] = sum(r["dB"] for r in res)
@@ -82,3 +121,32 @@ def batched_adjoint_grad(theta, x, g, tbar, **kw):
         else:
             res[k] = np.stack([o[k] for o in outs])
     return res
+
+
+def ssm_forward(theta, x, channel_block=64):
+    """`oracle.ssm_oracle.ssm_forward` with the channel blocks of the scan on worker processes."""
+    u, delta, Bm, Cm, A = O.nets(theta, x)
+    jobs = [(delta[:, p0:p0 + channel_block], x[:, p0:p0 + channel_block], Bm, Cm, A[p0:p0 + channel_block])
+            for p0 in range(0, x.shape[1], channel_block)]
+    res = map_bounded(_fwd_block, jobs, _scan_gb(x.shape[0], channel_block, A.shape[1]) / 2)
+    return np.concatenate(res, axis=1)
+
+
+def stack_grad(thetas, y0, g, tbar, mode="chained", store=None, channel_block=64):
+    """`oracle.ssm_oracle.stack_grad` (block tier) for one sequence with each layer's scans on worker processes: the
+    same sequence of oracle calls (rmsnorm, layer forward, adjoint_grad, rmsnorm_vjp) and the `store` hook at the same
+    places.  Returns ({"grads": per-layer dicts, "yK": top activation}, G_0 or None)."""
+    keep = (lambda a: a) if store is None else store
+    ys, yhats = [y0], []
+    for th in thetas:
+        yhats.append(keep(O.rmsnorm(ys[-1])))
+        ys.append(keep(ys[-1] + keep(ssm_forward(th, yhats[-1], channel_block))))
+    K = len(thetas)
+    grads = [None] * K
+    G = g
+    for k in range(K - 1, -1, -1):
+        grads[k] = adjoint_grad(thetas[k], yhats[k], G if mode == "chained" else g, tbar, tier="block",
+                                channel_block=channel_block)
+        if mode == "chained":
+            G = keep(G + O.rmsnorm_vjp(ys[k], keep(grads[k]["dx"])))
+    return {"grads": grads, "yK": ys[-1]}, (G if mode == "chained" else None)

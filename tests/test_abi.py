@@ -31,7 +31,7 @@ def test_exports_match_header(L):
 
 
 def test_version_and_strerror(L):
-    assert B.as_version() == 101
+    assert B.as_version() == 102
     assert B.strerror(0) == "ok"
     assert "tbar" in B.strerror(B.AS_ERR_TBAR)
     assert "unknown" in B.strerror(-999)
@@ -57,6 +57,12 @@ def test_workspace_query_and_argument_errors(L):
     with pytest.raises(B.AsError) as ei:
         B.as_workspace_bytes(sh, 0)
     assert ei.value.code == B.AS_ERR_TBAR
+    # sizes beyond the 32-bit token-row coordinates or the segment grid dimension are refused, not mis-addressed
+    for bad in (B.make_shape(4, 1 << 29, 64), B.make_shape(1, (1 << 31) - 64, 8), B.make_shape(1, 65536 * 2048, 8)):
+        with pytest.raises(B.AsError) as ei:
+            B.as_workspace_bytes(bad, 4)
+        assert ei.value.code == B.AS_ERR_LIMIT
+    assert B.as_sm_count() >= 1
     # NULL pointers are rejected before any CUDA call
     p = B.as_params_t(None, None, None, None, None)
     g = B.as_grads_t(None, None, None, None, None, None)

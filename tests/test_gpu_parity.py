@@ -8,7 +8,8 @@ from paper_2501_00692_b200 import binding as B
 from paper_2501_00692_b200 import synth
 from paper_2501_00692_b200.build import build_library
 
-from gpu_util import (TOL, assert_close, compare_grads, gpu_adjoint, gpu_forward, oracle_adjoint, theta_f64)
+from gpu_util import (TOL, assert_close, assert_dalog_rows, compare_all, compare_grads, gpu_adjoint, gpu_forward,
+                      oracle_adjoint, oracle_adjoint_with_bound, theta_f64)
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -135,16 +136,45 @@ def test_degenerate_and_tiny_shapes(batch, T, P, tbar, io):
     # bf16 widths that take the FP32-pipe contraction path (d_model not a multiple of 32)
     w = synth.custom_workload("tiny", 16, batch, T, P, tbar=tbar, io=io)
     theta, x, dy = setup(w, slow=True)
-    ref = oracle_adjoint(theta, x, dy, tbar, tier="direct")
-    # With a single token dA_log is identically zero (h_0 = 0).  The library forms abar_t h_{t-1} as
-    # h_t - Delta_t x_t B_t with one rounding, so its error is relative to |h_t|, not to the vanishing difference:
-    # measure it against the size of the other state-dependent gradient, dW_B.
-    zf = {"dA_log": float(np.abs(ref["dW_B"]).max())}
-    compare_grads(gpu_adjoint(w, theta, x, dy, tbar), ref, TOL[io], zero_floor=zf)
+    ref = oracle_adjoint_with_bound(theta, x, dy, tbar, tier="direct")
+    # With a single token dA_log is identically zero in the oracle (h_0 = 0); the library's value is then pure
+    # rounding of h_1 - Delta_1 x_1 B_1 and must stay inside the row-wise bound built from the oracle's own mu and h.
+    compare_all(gpu_adjoint(w, theta, x, dy, tbar), ref, TOL[io])
     y = gpu_forward(w, theta, x)
     assert_close(synth.to_f64(y), ref["y"], TOL[io], "y")
     gb = gpu_adjoint(w, theta, x, dy, T, bptt=True)
     compare_grads(gb, oracle_adjoint(theta, x, dy, T, tier="direct"), TOL[io])
+
+
+@pytest.mark.parametrize("io", ["f32", "bf16"])
+@pytest.mark.parametrize("law", ["fast", "standard", "slow"])
+@pytest.mark.parametrize("T", [2, 3, 8, 64, 300])
+def test_dalog_row_by_row(T, law, io):
+    """dA_log channel by channel where abar_i h_{i-1} is small against h_i: very short sequences (h_{i-1} is zero or
+    one step old) and the fast-decay corner b_delta ~ U(-1, 1) (abar << 1).  The library forms abar_i h_{i-1} as
+    h_i - Delta_i x_i B_i; the bound allows DALOG_C rounding units of h_i per term beyond the tolerance and the test
+    reports how much of that allowance was used."""
+    w = synth.custom_workload("dalog", 18, 2, T, 72, tbar=max(1, T // 2), io=io)
+    rng = {"fast": (-1.0, 1.0), "standard": None, "slow": (-9.0, -7.0)}[law]
+    theta = synth.layer_params(w, 0, DEV, b_delta_range=rng)
+    x, dy = synth.activations(w, DEV)
+    for tbar in (w.tbar, T):
+        ref = oracle_adjoint_with_bound(theta, x, dy, tbar, tier="direct")
+        g = gpu_adjoint(w, theta, x, dy, tbar)
+        use = assert_dalog_rows(synth.to_f64(g["dA_log"]), ref, TOL[io])
+        compare_grads(g, ref, TOL[io], keys=("dW_delta", "db_delta", "dW_B", "dW_C", "dx"))
+        print(f"dA_log rows T={T} law={law} io={io} tbar={tbar}: {use}")
+
+
+def test_bptt_comparator_bf16_multi_segment():
+    """as_full_bptt_grad on bf16 I/O over several of its 64-token checkpoint segments and time segments."""
+    w = synth.custom_workload("bptt16", 19, 2, 4100, 160, io="bf16")
+    theta, x, dy = setup(w, slow=True)
+    ref = O.batched(O.bptt_grad, theta_f64(theta), synth.to_f64(x), synth.to_f64(dy))
+    gb = gpu_adjoint(w, theta, x, dy, w.seqlen, bptt=True)
+    compare_grads(gb, ref, TOL["bf16"])
+    ga = gpu_adjoint(w, theta, x, dy, w.seqlen)
+    compare_grads(ga, ref, TOL["bf16"])
 
 
 def test_zero_upstream_gradient_gives_zero():

@@ -373,3 +373,22 @@ def test_parallel_harness_equals_adjoint_grad():
         for k in GRADS + ("y",):
             assert np.abs(got[k] - ref[k]).max() <= 1e-13 * (np.abs(ref[k]).max() + 1e-300), (tier, k)
         assert got["absq"].shape == (P, N) and (got["absq"] >= 0).all()
+
+
+def test_parallel_stack_harness_equals_stack_grad():
+    import oracle_parallel as OP
+    from gpu_util import bf16_round
+    rng = np.random.default_rng(5)
+    P, N, T, K = 12, 16, 40, 3
+    ths = [make_theta(rng, P, N) for _ in range(K)]
+    y0, g = rng.normal(size=(T, P)), rng.normal(size=(T, P))
+    for mode in ("chained", "paper"):
+        for store in (None, bf16_round):
+            a, Ga = O.stack_grad(ths, y0, g, 7, mode=mode, tier="block", store=store)
+            b, Gb = OP.stack_grad(ths, y0, g, 7, mode, store, channel_block=5)
+            for k in range(K):
+                for name in O.PARAM_GRADS:
+                    assert np.abs(a[k][name] - b["grads"][k][name]).max() <= 1e-12 * np.abs(a[k][name]).max()
+            if mode == "chained":
+                assert np.abs(Ga - Gb).max() <= 1e-12 * np.abs(Ga).max()
+            assert np.abs(b["yK"] - O.stack_forward(ths, y0, store)[0][-1]).max() <= 1e-12

@@ -40,6 +40,8 @@ def test_static_scratch_forward_matches_regular_forward_twice(io):
         stream = C.c_void_p(torch.cuda.current_stream().cuda_stream)
         rc = L.as_ssm_forward_static(C.byref(sh), C.byref(p), C.c_void_p(x.data_ptr()), C.c_void_p(y.data_ptr()), stream)
         assert rc == 0, B.strerror(rc)
+        # the status word of this entry point's kernels sits in the built-in array: NULL selects it
+        assert L.as_check_status(None, stream) == B.AS_OK
         torch.cuda.synchronize()
         assert torch.isfinite(y.float()).all()
         tol = 1e-4 if io == "f32" else 2e-2
