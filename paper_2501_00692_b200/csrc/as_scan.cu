@@ -35,7 +35,7 @@ int make_plan(const as_shape_t* sh, int64_t tbar, Plan* pl) {
   p.bw = p.P < CH ? p.P : CH;
   const int64_t ctas = (int64_t)p.tiles * p.B;
   // two full waves of the main kernel's resident CTAs (148 SMs x CTAs per SM), never more than that
-  const int64_t slots = (int64_t)sm_count() * 3;
+  const int64_t slots = (int64_t)sm_count() * AS_MAIN_CTAS;
   int64_t s_target = (2 * slots) / ctas;
   if (s_target < 1) s_target = 1;
   int64_t L = (p.T + s_target - 1) / s_target;
@@ -156,9 +156,22 @@ struct Stage {
 };
 constexpr int NSTAGE = 3;        // ascending kernels
 constexpr int WRED_Q = 32 * 4 + 8;   // floats per quarter-block of the per-warp reduction scratch (512 B + 32 B skew)
-constexpr int MAIN_CTAS = 3;    // resident CTAs per SM the main kernel is compiled for (up to 168 registers per thread)
-constexpr int FW_UNROLL = 4;     // unroll factor of the main adjoint kernel's forward rebuild loop
-constexpr int BW_UNROLL = 2;     // unroll factor of the main adjoint kernel's backward token loop
+#ifndef AS_MAIN_CTAS
+#define AS_MAIN_CTAS 3
+#endif
+#ifndef AS_PARK_ABAR
+#define AS_PARK_ABAR 0
+#endif
+constexpr int MAIN_CTAS = AS_MAIN_CTAS;    // resident CTAs per SM the main kernel is compiled for
+constexpr bool PARK_ABAR = AS_PARK_ABAR != 0;   // park abar_j next to h_j in tensor memory: the backward walk then needs no ex2
+#ifndef AS_FW_UNROLL
+#define AS_FW_UNROLL 4
+#endif
+#ifndef AS_BW_UNROLL
+#define AS_BW_UNROLL 2
+#endif
+constexpr int FW_UNROLL = AS_FW_UNROLL;     // unroll factor of the main adjoint kernel's forward rebuild loop
+constexpr int BW_UNROLL = AS_BW_UNROLL;     // unroll factor of the main adjoint kernel's backward token loop
 constexpr int NSTAGE_MAIN = 2;   // main adjoint kernel: a chunk takes thousands of cycles, one chunk of lookahead suffices
 
 // per-thread values of its NCH channels
@@ -617,7 +630,8 @@ __device__ __forceinline__ void decay_units(const u64 (&e2)[NCH], const u64 (&A2
 // columns of its SM (three CTAs are resident) and every thread parks the chunk's eight states in its own TMEM lane:
 // warp w of the 4-warp CTA owns lanes [32w, 32w+32), a 32x32b access moves 16 registers of each lane to or
 // from 16 consecutive columns.
-constexpr int TM_COLS = CK * 16;   // columns [16 j, 16 j + 16): state after token j of the current chunk
+constexpr int TM_TOK = PARK_ABAR ? 32 : 16;   // columns per token: h_j (16) and, when parked, abar_j (16)
+constexpr int TM_COLS = CK * TM_TOK;
 
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const u64 (&v)[NU]) {
   uint32_t r[16];
@@ -641,6 +655,28 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, u64 (&v)[NU]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
   for (int u = 0; u < 8; ++u) asm("mov.b64 %0, {%1, %2};" : "=l"(v[u]) : "r"(r[2 * u]), "r"(r[2 * u + 1]));
+}
+// two 16-column loads behind one wait
+__device__ __forceinline__ void tmem_ld16x2(uint32_t taddr, u64 (&v)[NU], u64 (&w2)[NU]) {
+  uint32_t r[16], q[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(q[0]), "=r"(q[1]), "=r"(q[2]), "=r"(q[3]), "=r"(q[4]), "=r"(q[5]), "=r"(q[6]), "=r"(q[7]), "=r"(q[8]),
+        "=r"(q[9]), "=r"(q[10]), "=r"(q[11]), "=r"(q[12]), "=r"(q[13]), "=r"(q[14]), "=r"(q[15])
+      : "r"(taddr + 16)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int u = 0; u < 8; ++u) {
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v[u]) : "r"(r[2 * u]), "r"(r[2 * u + 1]));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(w2[u]) : "r"(q[2 * u]), "r"(q[2 * u + 1]));
+  }
 }
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -886,7 +922,8 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
           decay_units<SC>(d2, A2, af);
 #pragma unroll
           for (int u = 0; u < NU; ++u) h[u] = fma2(af[u], h[u], mul2(dx2[u / 4], Bp[u % 4]));
-          tmem_st16(tm + 16 * j, h);
+          tmem_st16(tm + TM_TOK * j, h);
+          if (PARK_ABAR) tmem_st16(tm + TM_TOK * j + 16, af);
         }
         tmem_wait_st();
       }
@@ -904,12 +941,13 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
       const uint8_t* pX = sm + St::X + (CK - 1) * CH * ESZ + ESZ * NCH * w.k;   // x row; dy row at + (St::G - St::X)
       const float* pB = reinterpret_cast<const float*>(sm + St::BC) + 8 * w.half + (CK - 1) * NBC;   // [B | C] row
       float* pR = &red[rb][warp][CK - 1][((lane >> 1) & 8) * 2 + 8 * w.half + ((lane >> 1) & 7)];
-      uint32_t tmj = tm + 16 * (CK - 1);
+      uint32_t tmj = tm + TM_TOK * (CK - 1);
 #pragma unroll BW_UNROLL
       for (int j = CK - 1; j >= 0; --j) {
-        u64 hT[NU];
-        tmem_ld16(tmj, hT);
-        tmj -= 16;
+        u64 hT[NU], aT[NU];
+        if (PARK_ABAR) tmem_ld16x2(tmj, hT, aT);
+        else tmem_ld16(tmj, hT);
+        tmj -= TM_TOK;
         const ChV dv = lds_chp<float>(pD);
         const ChV xv = lds_chp<IO>(pX);
         const ChV gv = lds_chp<IO>(pX + (St::G - St::X));
@@ -963,11 +1001,11 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         for (int ch = 0; ch < NCH; ++ch) {
           u64 sacc, dacc;
           u64 ach = 0ull;
-          if (SC) ach = ex2_2(mul2(d2[ch], A2[ch * 4]));   // scalar rate: one factor for the channel's states
+          if (SC && !PARK_ABAR) ach = ex2_2(mul2(d2[ch], A2[ch * 4]));   // scalar rate: one factor for the channel's states
 #pragma unroll
           for (int m = 0; m < 4; ++m) {
             const int u = ch * 4 + m;
-            const u64 a = SC ? ach : ex2_2(mul2(d2[ch], A2[u]));
+            const u64 a = PARK_ABAR ? aT[u] : (SC ? ach : ex2_2(mul2(d2[ch], A2[u])));
             const u64 hn = hT[u];                                  // h_i
             const u64 hb = fma2(ndx2[ch], Bp[m], hn);              // abar_i h_{i-1} = h_i - Delta_i x_i B_i
             vB[m] = ch == 0 ? mul2(mu[u], dx2[ch]) : fma2(mu[u], dx2[ch], vB[m]);   // dB partial (two channels)
