@@ -43,7 +43,7 @@
 extern "C" {
 #endif
 
-#define AS_VERSION 102
+#define AS_VERSION 103
 
 typedef enum { AS_F32 = 0, AS_BF16 = 1 } as_dtype_t;
 
@@ -83,6 +83,9 @@ typedef struct {          /* parameters of one layer (device pointers) */
   const void  *W_B;       /* [N,P] io dtype */
   const void  *W_C;       /* [N,P] io dtype */
   const float *A_log;     /* [P,N] fp32 (AS_A_SCALAR: [P]), A = -exp(A_log) */
+  const void  *Wcat;      /* optional, may be NULL: [P+32, P] io dtype, the rows of W_delta, W_B, W_C stacked, as written
+                             by as_pack_weights.  Only the bf16 tensor-core contractions read it (bf16 io, P % 32 == 0);
+                             when NULL they pack a copy into the scratch on every call (one more small kernel). */
 } as_params_t;
 
 typedef struct {          /* gradient outputs (device pointers); parameter gradients are fp32, summed over the batch */
@@ -127,6 +130,36 @@ int as_ssm_forward(const as_shape_t *shape, const as_params_t *params, const voi
 int as_adjoint_grad(const as_shape_t *shape, const as_params_t *params, const void *x, const void *dy,
                     int64_t tbar, uint32_t flags, const as_grads_t *out,
                     void *ws, size_t ws_bytes, void *stream);
+
+/* The K layers of a residual stack in one call (Proposition 3 and Section 4.2: given the stored layer inputs and the
+ * one upstream gradient dL/dy_K, the adjoint states of a layer depend only on that layer's own A and C, so all
+ * layers' vector-Jacobian products are independent; Alg. 4's loop over k).  Every phase - projections, segment
+ * pre-pass, carries, main adjoint kernel, the two contractions - runs as ONE launch over (layer, batch element)
+ * instead of one launch per layer.
+ *   layers  K >= 1;
+ *   params  every pointer addresses K contiguous copies of the single-layer tensor: W_delta [K,P,P], b_delta [K,P],
+ *           W_B, W_C [K,N,P], A_log [K,P,N] ([K,P] for AS_A_SCALAR), Wcat [K,P+32,P] or NULL;
+ *   x       [K,Bsz,T,P] io: the input of each layer (for the stack: Norm(y_{k-1}));
+ *   dy      [Bsz,T,P] io: shared by all layers;
+ *   out     every pointer addresses K contiguous copies: dW_delta [K,P,P], ..., dA_log [K,P,N]; dx [K,Bsz,T,P] or NULL;
+ *   ws      at least as_workspace_bytes_layers bytes.
+ * Layer k's results equal as_adjoint_grad on (params[k], x[k], dy).  The bf16 contractions go out as one launch when
+ * Bsz*T is a multiple of 128 (no 128-row tile then straddles two layers), otherwise as one launch per layer; fp32 io
+ * runs its FP32-pipe contractions layer by layer.  K = 1 is exactly as_adjoint_grad.
+ * Limits: K * Bsz <= 65535 and K * Bsz * T + T + 16 < 2^31 (AS_ERR_LIMIT). */
+int as_adjoint_grad_layers(const as_shape_t *shape, int32_t layers, const as_params_t *params, const void *x,
+                           const void *dy, int64_t tbar, uint32_t flags, const as_grads_t *out,
+                           void *ws, size_t ws_bytes, void *stream);
+
+/* Scratch size of as_adjoint_grad_layers. */
+int as_workspace_bytes_layers(const as_shape_t *shape, int32_t layers, int64_t tbar, size_t *grad_bytes);
+
+/* Packed weights for the bf16 tensor-core contractions: Wcat[k] = [W_delta[k]; W_B[k]; W_C[k]], [layers, P+32, P].
+ * as_wcat_bytes gives the buffer size (0 for a bad shape); as_pack_weights writes it (bf16 io only, AS_ERR_DTYPE
+ * otherwise).  Pack once per parameter update and pass the pointer as as_params_t.Wcat: the forward and gradient
+ * calls then skip their own packing kernel.  The packed copy must be re-made whenever W_delta, W_B or W_C change. */
+size_t as_wcat_bytes(const as_shape_t *shape, int32_t layers);
+int as_pack_weights(const as_shape_t *shape, int32_t layers, const as_params_t *params, void *wcat, void *stream);
 
 /* The same outputs by plain backpropagation through time (the sequential nested accumulation that the
  * adjoint method replaces, Section 3.3): one reverse sweep per channel carrying dL/dh_t.  Separately coded

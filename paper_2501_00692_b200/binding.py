@@ -23,7 +23,8 @@ AS_ERR_WORKSPACE, AS_ERR_ALIGN, AS_ERR_CUDA, AS_ERR_TIMEOUT, AS_ERR_LIMIT = -5, 
 
 EXPORTS = ("as_version", "as_strerror", "as_workspace_bytes", "as_check_status", "as_ssm_forward",
            "as_adjoint_grad", "as_full_bptt_grad", "as_rmsnorm_fwd", "as_residual_add", "as_rmsnorm_bwd_add",
-           "as_launch_count", "as_set_timing", "as_get_timing", "as_ssm_forward_static", "as_wait_selftest", "as_sm_count")
+           "as_launch_count", "as_set_timing", "as_get_timing", "as_ssm_forward_static", "as_wait_selftest", "as_sm_count",
+           "as_adjoint_grad_layers", "as_workspace_bytes_layers", "as_wcat_bytes", "as_pack_weights")
 AS_STATIC_SCRATCH_BYTES = 32 << 20
 AS_NUM_PHASES = 6
 PHASES = ("projections", "prepass", "fixup", "adjoint_main", "weight_grads", "input_grad")
@@ -36,7 +37,7 @@ class as_shape_t(C.Structure):
 
 class as_params_t(C.Structure):
     _fields_ = [("W_delta", C.c_void_p), ("b_delta", C.c_void_p), ("W_B", C.c_void_p),
-                ("W_C", C.c_void_p), ("A_log", C.c_void_p)]
+                ("W_C", C.c_void_p), ("A_log", C.c_void_p), ("Wcat", C.c_void_p)]
 
 
 class as_grads_t(C.Structure):
@@ -79,13 +80,20 @@ def lib() -> C.CDLL:
         L.as_ssm_forward_static.argtypes = [C.POINTER(as_shape_t), C.POINTER(as_params_t), C.c_void_p, C.c_void_p,
                                             C.c_void_p]
         L.as_wait_selftest.argtypes = [C.c_void_p, C.c_size_t, C.c_uint32, C.c_void_p]
+        L.as_adjoint_grad_layers.argtypes = [C.POINTER(as_shape_t), C.c_int32, C.POINTER(as_params_t), C.c_void_p,
+                                             C.c_void_p, C.c_int64, C.c_uint32, C.POINTER(as_grads_t), C.c_void_p,
+                                             C.c_size_t, C.c_void_p]
+        L.as_workspace_bytes_layers.argtypes = [C.POINTER(as_shape_t), C.c_int32, C.c_int64, C.POINTER(C.c_size_t)]
+        L.as_wcat_bytes.argtypes = [C.POINTER(as_shape_t), C.c_int32]
+        L.as_pack_weights.argtypes = [C.POINTER(as_shape_t), C.c_int32, C.POINTER(as_params_t), C.c_void_p, C.c_void_p]
         L.as_launch_count.argtypes = [C.c_int]
         L.as_set_timing.argtypes = [C.c_int]
         L.as_get_timing.argtypes = [C.POINTER(C.c_float), C.c_int]
         for name in EXPORTS:
-            if name not in ("as_strerror", "as_launch_count"):
+            if name not in ("as_strerror", "as_launch_count", "as_wcat_bytes"):
                 getattr(L, name).restype = C.c_int
         L.as_launch_count.restype = C.c_int64
+        L.as_wcat_bytes.restype = C.c_size_t
         _lib = L
     return _lib
 
@@ -115,7 +123,8 @@ def shape_of(x: torch.Tensor, d_state=16, a_scalar=False) -> as_shape_t:
 
 
 def make_params(theta: dict) -> as_params_t:
-    return as_params_t(*[_ptr(theta[k]) for k in ("W_delta", "b_delta", "W_B", "W_C", "A_log")])
+    """theta may carry an optional "Wcat" (the packed weights of as_pack_weights)."""
+    return as_params_t(*[_ptr(theta[k]) for k in ("W_delta", "b_delta", "W_B", "W_C", "A_log")], _ptr(theta.get("Wcat")))
 
 
 def alloc_grads(shape: as_shape_t, device, with_dx=True) -> dict:
@@ -176,6 +185,43 @@ def as_adjoint_grad(shape, theta, x, dy, tbar, grads, ws, flags=0, stream=None):
     p, g = make_params(theta), make_grads(grads)
     _check(lib().as_adjoint_grad(C.byref(shape), C.byref(p), _ptr(x), _ptr(dy), int(tbar), int(flags), C.byref(g),
                                  _ptr(ws), ws.numel(), _stream(stream)), "as_adjoint_grad")
+
+
+def as_workspace_bytes_layers(shape: as_shape_t, layers: int, tbar: int) -> int:
+    grad = C.c_size_t(0)
+    _check(lib().as_workspace_bytes_layers(C.byref(shape), int(layers), int(tbar), C.byref(grad)),
+           "as_workspace_bytes_layers")
+    return grad.value
+
+
+def as_adjoint_grad_layers(shape, layers, theta, x, dy, tbar, grads, ws, flags=0, stream=None):
+    """All layers of a stack in one call: every tensor of `theta` and `grads` has a leading [layers] dimension,
+    x is [layers, B, T, P], dy [B, T, P] is shared."""
+    p, g = make_params(theta), make_grads(grads)
+    _check(lib().as_adjoint_grad_layers(C.byref(shape), int(layers), C.byref(p), _ptr(x), _ptr(dy), int(tbar), int(flags),
+                                        C.byref(g), _ptr(ws), ws.numel(), _stream(stream)), "as_adjoint_grad_layers")
+
+
+def as_wcat_bytes(shape: as_shape_t, layers: int = 1) -> int:
+    return int(lib().as_wcat_bytes(C.byref(shape), int(layers)))
+
+
+def as_pack_weights(shape, layers, theta, wcat, stream=None):
+    p = make_params(theta)
+    _check(lib().as_pack_weights(C.byref(shape), int(layers), C.byref(p), _ptr(wcat), _stream(stream)), "as_pack_weights")
+
+
+def alloc_grads_layers(shape: as_shape_t, layers: int, device, with_dx=False) -> dict:
+    """Gradient buffers with a leading [layers] dimension for as_adjoint_grad_layers."""
+    P, N, K = shape.d_model, shape.d_state, int(layers)
+    f = dict(dtype=torch.float32, device=device)
+    g = {"dW_delta": torch.empty(K, P, P, **f), "db_delta": torch.empty(K, P, **f), "dW_B": torch.empty(K, N, P, **f),
+         "dW_C": torch.empty(K, N, P, **f),
+         "dA_log": torch.empty(K, P, **f) if shape.a_structure == AS_A_SCALAR else torch.empty(K, P, N, **f), "dx": None}
+    if with_dx:
+        dt = torch.float32 if shape.io == AS_F32 else torch.bfloat16
+        g["dx"] = torch.empty(K, shape.batch, shape.seqlen, P, dtype=dt, device=device)
+    return g
 
 
 def as_full_bptt_grad(shape, theta, x, dy, grads, ws, flags=0, stream=None):

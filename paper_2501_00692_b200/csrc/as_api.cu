@@ -40,7 +40,7 @@ int check_shape(const as_shape_t* sh) {
 int check_params(const as_params_t* pr) {
   if (!pr || !pr->W_delta || !pr->b_delta || !pr->W_B || !pr->W_C || !pr->A_log) return AS_ERR_NULL;
   if (!aligned16(pr->W_delta) || !aligned16(pr->b_delta) || !aligned16(pr->W_B) || !aligned16(pr->W_C) ||
-      !aligned16(pr->A_log))
+      !aligned16(pr->A_log) || !aligned16(pr->Wcat))
     return AS_ERR_ALIGN;
   return AS_OK;
 }
@@ -51,27 +51,39 @@ int check_params(const as_params_t* pr) {
     if (e__ != 0) return AS_ERR_CUDA;     \
   } while (0)
 
-// steps 1-3 of SSM(.): Delta = softplus(x W_delta^T + b), B = x W_B^T, C = x W_C^T
-int projections(const Plan& pl, const as_params_t* pr, const void* x, char* ws, cudaStream_t st) {
+// Wcat of the call: the caller's packed copy if it gave one, else packed here into the scratch
+int wcat_of(const Plan& pl, const as_params_t* pr, char* ws, cudaStream_t st, const void** wcat) {
+  if (pr->Wcat) { *wcat = pr->Wcat; return AS_OK; }
+  AS_TRY(tc_pack_wcat(pl.P, pl.KL, pr, ws + pl.off_wcat, st));
+  *wcat = ws + pl.off_wcat;
+  return AS_OK;
+}
+
+// steps 1-3 of SSM(.): Delta = softplus(x W_delta^T + b), B = x W_B^T, C = x W_C^T  (every layer of the call)
+int projections(const Plan& pl, const as_params_t* pr, const void* wcat, const void* x, char* ws, cudaStream_t st) {
   if (pl.tc) {
-    AS_TRY(tc_pack_wcat(pl, pr, ws, st));
-    AS_TRY(tc_projections(pl, pr, x, ws, st));
+    AS_TRY(tc_projections(pl, pr, wcat, x, ws, st));
     return AS_OK;
   }
   const int bf = pl.io == AS_BF16;
-  const int64_t M = (int64_t)pl.B * pl.T;
-  GemmArgs g{};
-  g.A = x; g.a_bf16 = bf; g.a_sm = pl.P; g.a_sk = 1;
-  g.b_bf16 = bf; g.b_sn = pl.P; g.b_sk = 1;
-  g.M = M; g.K = pl.P; g.splitk = 1;
-  g.Bm = pr->W_delta; g.N = pl.P; g.C = reinterpret_cast<float*>(ws + pl.off_delta); g.ldc = pl.P; g.coff = 0;
-  g.bias = pr->b_delta; g.epi = EPI_SOFTPLUS_BIAS;
-  AS_TRY(launch_gemm_simt(g, st));
-  g.epi = EPI_STORE; g.bias = nullptr; g.N = NS; g.C = reinterpret_cast<float*>(ws + pl.off_bc); g.ldc = NBC;
-  g.Bm = pr->W_B; g.coff = 0;
-  AS_TRY(launch_gemm_simt(g, st));
-  g.Bm = pr->W_C; g.coff = NS;
-  AS_TRY(launch_gemm_simt(g, st));
+  const size_t e = bf ? 2 : 4;
+  const int64_t M = (int64_t)pl.Bg * pl.T;
+  const size_t P = pl.P;
+  for (int l = 0; l < pl.KL; ++l) {
+    GemmArgs g{};
+    g.A = (const char*)x + l * M * P * e; g.a_bf16 = bf; g.a_sm = pl.P; g.a_sk = 1;
+    g.b_bf16 = bf; g.b_sn = pl.P; g.b_sk = 1;
+    g.M = M; g.K = pl.P; g.splitk = 1;
+    g.Bm = (const char*)pr->W_delta + l * P * P * e; g.N = pl.P;
+    g.C = reinterpret_cast<float*>(ws + pl.off_delta) + l * M * P; g.ldc = pl.P; g.coff = 0;
+    g.bias = pr->b_delta + l * P; g.epi = EPI_SOFTPLUS_BIAS;
+    AS_TRY(launch_gemm_simt(g, st));
+    g.epi = EPI_STORE; g.bias = nullptr; g.N = NS; g.C = reinterpret_cast<float*>(ws + pl.off_bc) + l * M * NBC; g.ldc = NBC;
+    g.Bm = (const char*)pr->W_B + l * NS * P * e; g.coff = 0;
+    AS_TRY(launch_gemm_simt(g, st));
+    g.Bm = (const char*)pr->W_C + l * NS * P * e; g.coff = NS;
+    AS_TRY(launch_gemm_simt(g, st));
+  }
   return AS_OK;
 }
 
@@ -84,50 +96,57 @@ int pick_splitk(int64_t tiles, int64_t K) {
   return (int)s;
 }
 
-// the net-VJPs: weight gradients (contractions over all tokens) and the input gradient
-int contractions(const Plan& pl, const as_params_t* pr, const void* x, const as_grads_t* out, char* ws,
+// the net-VJPs: weight gradients (contractions over all tokens) and the input gradient, for every layer of the call
+int contractions(const Plan& pl, const as_params_t* pr, const void* wcat, const void* x, const as_grads_t* out, char* ws,
                  cudaStream_t st) {
   const int bf = pl.io == AS_BF16;
-  const int64_t M = (int64_t)pl.B * pl.T;
+  const size_t e = bf ? 2 : 4;
+  const int64_t M = (int64_t)pl.Bg * pl.T;
   const int P = pl.P;
-  const void* du = ws + pl.off_du;
-  const float* dbc = reinterpret_cast<const float*>(ws + pl.off_dbc);
   if (pl.tc) {
     AS_TRY(tc_weight_grads(pl, x, out, ws, st));
     mark(5, st);
-    if (out->dx) AS_TRY(tc_input_grad(pl, out->dx, ws, st));
+    if (out->dx) AS_TRY(tc_input_grad(pl, wcat, out->dx, ws, st));
     mark(6, st);
     return AS_OK;
   }
-  {  // dW_delta[i,j] = sum_m du[m,i] x[m,j]
+  for (int l = 0; l < pl.KL; ++l) {
+    const void* du = ws + pl.off_du + (size_t)l * M * pl.du_ld * e;
+    const float* dbc = reinterpret_cast<const float*>(ws + pl.off_dbc) + (size_t)l * M * NBC;
+    const void* xl = (const char*)x + (size_t)l * M * P * e;
+    // dW_delta[i,j] = sum_m du[m,i] x[m,j]
     GemmArgs g{};
     g.A = du; g.a_bf16 = bf; g.a_sm = 1; g.a_sk = P;
-    g.Bm = x; g.b_bf16 = bf; g.b_sn = 1; g.b_sk = P;
-    g.C = out->dW_delta; g.ldc = P; g.coff = 0; g.M = P; g.N = P; g.K = M; g.epi = EPI_ATOMIC;
+    g.Bm = xl; g.b_bf16 = bf; g.b_sn = 1; g.b_sk = P;
+    g.C = out->dW_delta + (size_t)l * P * P; g.ldc = P; g.coff = 0; g.M = P; g.N = P; g.K = M; g.epi = EPI_ATOMIC;
     g.splitk = pick_splitk((int64_t)((P + 63) / 64) * ((P + 63) / 64), M);
     AS_TRY(launch_gemm_simt(g, st));
     // dW_B, dW_C
     g.A = dbc; g.a_bf16 = 0; g.a_sm = 1; g.a_sk = NBC; g.M = NS;
     g.splitk = pick_splitk((P + 63) / 64, M);
-    g.C = out->dW_B;
+    g.C = out->dW_B + (size_t)l * NS * P;
     AS_TRY(launch_gemm_simt(g, st));
-    g.A = dbc + NS; g.C = out->dW_C;
+    g.A = dbc + NS; g.C = out->dW_C + (size_t)l * NS * P;
     AS_TRY(launch_gemm_simt(g, st));
   }
   mark(5, st);
   if (out->dx) {  // dx = dx_dir + du W_delta + dB W_B + dC W_C
-    float* acc = reinterpret_cast<float*>(ws + pl.off_dxacc);
-    GemmArgs g{};
-    g.A = du; g.a_bf16 = bf; g.a_sm = P; g.a_sk = 1;
-    g.Bm = pr->W_delta; g.b_bf16 = bf; g.b_sn = 1; g.b_sk = P;
-    g.C = acc; g.ldc = P; g.coff = 0; g.M = M; g.N = P; g.K = P; g.epi = EPI_STORE; g.splitk = 1;
-    AS_TRY(launch_gemm_simt(g, st));
-    g.A = dbc; g.a_bf16 = 0; g.a_sm = NBC; g.a_sk = 1; g.K = NS; g.epi = EPI_ACCUM;
-    g.Bm = pr->W_B;
-    AS_TRY(launch_gemm_simt(g, st));
-    g.A = dbc + NS; g.Bm = pr->W_C;
-    AS_TRY(launch_gemm_simt(g, st));
-    AS_TRY(launch_finish_dx(pl, acc, ws + pl.off_dxdir, out->dx, st));
+    for (int l = 0; l < pl.KL; ++l) {
+      const void* du = ws + pl.off_du + (size_t)l * M * pl.du_ld * e;
+      const float* dbc = reinterpret_cast<const float*>(ws + pl.off_dbc) + (size_t)l * M * NBC;
+      float* acc = reinterpret_cast<float*>(ws + pl.off_dxacc) + (size_t)l * M * P;
+      GemmArgs g{};
+      g.A = du; g.a_bf16 = bf; g.a_sm = P; g.a_sk = 1;
+      g.Bm = (const char*)pr->W_delta + (size_t)l * P * P * e; g.b_bf16 = bf; g.b_sn = 1; g.b_sk = P;
+      g.C = acc; g.ldc = P; g.coff = 0; g.M = M; g.N = P; g.K = P; g.epi = EPI_STORE; g.splitk = 1;
+      AS_TRY(launch_gemm_simt(g, st));
+      g.A = dbc; g.a_bf16 = 0; g.a_sm = NBC; g.a_sk = 1; g.K = NS; g.epi = EPI_ACCUM;
+      g.Bm = (const char*)pr->W_B + (size_t)l * NS * P * e;
+      AS_TRY(launch_gemm_simt(g, st));
+      g.A = dbc + NS; g.Bm = (const char*)pr->W_C + (size_t)l * NS * P * e;
+      AS_TRY(launch_gemm_simt(g, st));
+    }
+    AS_TRY(launch_finish_dx(pl, reinterpret_cast<const float*>(ws + pl.off_dxacc), ws + pl.off_dxdir, out->dx, st));
   }
   mark(6, st);
   return AS_OK;
@@ -148,15 +167,15 @@ int check_grad_args(const as_shape_t* sh, const as_params_t* pr, const void* x, 
 }
 
 int zero_outputs(const Plan& pl, uint32_t flags, const as_grads_t* out, char* ws, cudaStream_t st) {
-  const size_t P = pl.P;
+  const size_t P = pl.P, K = pl.KL;
   AS_TRY((int)cudaMemsetAsync(ws + pl.off_status, 0, 256, st));
   AS_TRY((int)cudaMemsetAsync(ws + pl.off_dbc, 0, (size_t)pl.B * pl.T * NBC * 4, st));
   if (!(flags & AS_ACCUMULATE)) {
-    AS_TRY((int)cudaMemsetAsync(out->dW_delta, 0, P * P * 4, st));
-    AS_TRY((int)cudaMemsetAsync(out->db_delta, 0, P * 4, st));
-    AS_TRY((int)cudaMemsetAsync(out->dW_B, 0, NS * P * 4, st));
-    AS_TRY((int)cudaMemsetAsync(out->dW_C, 0, NS * P * 4, st));
-    AS_TRY((int)cudaMemsetAsync(out->dA_log, 0, (pl.scalar ? P : P * NS) * 4, st));
+    AS_TRY((int)cudaMemsetAsync(out->dW_delta, 0, K * P * P * 4, st));
+    AS_TRY((int)cudaMemsetAsync(out->db_delta, 0, K * P * 4, st));
+    AS_TRY((int)cudaMemsetAsync(out->dW_B, 0, K * NS * P * 4, st));
+    AS_TRY((int)cudaMemsetAsync(out->dW_C, 0, K * NS * P * 4, st));
+    AS_TRY((int)cudaMemsetAsync(out->dA_log, 0, K * (pl.scalar ? P : P * NS) * 4, st));
   }
   return AS_OK;
 }
@@ -188,7 +207,7 @@ int as_workspace_bytes(const as_shape_t* shape, int64_t tbar, size_t* fwd_bytes,
   if (e) return e;
   if (tbar < 1) return AS_ERR_TBAR;
   Plan pl;
-  e = make_plan(shape, tbar, &pl);
+  e = make_plan(shape, tbar, 1, &pl);
   if (e) return e;
   if (fwd_bytes) *fwd_bytes = pl.total_fwd;
   if (grad_bytes) *grad_bytes = pl.total_grad;
@@ -218,13 +237,15 @@ int as_ssm_forward(const as_shape_t* shape, const as_params_t* params, const voi
   if (!x || !y || !ws) return AS_ERR_NULL;
   if (!aligned16(x) || !aligned16(y) || !aligned16(ws)) return AS_ERR_ALIGN;
   Plan pl;
-  e = make_plan(shape, shape->seqlen, &pl);
+  e = make_plan(shape, shape->seqlen, 1, &pl);
   if (e) return e;
   if (ws_bytes < pl.total_fwd) return AS_ERR_WORKSPACE;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   char* w = reinterpret_cast<char*>(ws);
   AS_TRY((int)cudaMemsetAsync(w + pl.off_status, 0, 256, st));
-  e = projections(pl, params, x, w, st);
+  const void* wcat = nullptr;
+  if (pl.tc) { e = wcat_of(pl, params, w, st, &wcat); if (e) return e; }
+  e = projections(pl, params, wcat, x, w, st);
   if (e) return e;
   ScanPtrs sp{x, nullptr, params->A_log, w};
   AS_TRY(launch_prepass(pl, sp, false, st));
@@ -235,11 +256,50 @@ int as_ssm_forward(const as_shape_t* shape, const as_params_t* params, const voi
 
 int as_adjoint_grad(const as_shape_t* shape, const as_params_t* params, const void* x, const void* dy, int64_t tbar,
                     uint32_t flags, const as_grads_t* out, void* ws, size_t ws_bytes, void* stream) {
+  return as_adjoint_grad_layers(shape, 1, params, x, dy, tbar, flags, out, ws, ws_bytes, stream);
+}
+
+int as_workspace_bytes_layers(const as_shape_t* shape, int32_t layers, int64_t tbar, size_t* grad_bytes) {
+  int e = check_shape(shape);
+  if (e) return e;
+  if (tbar < 1) return AS_ERR_TBAR;
+  if (layers < 1) return AS_ERR_SHAPE;
+  if ((int64_t)layers * shape->batch * shape->seqlen + shape->seqlen + 2 * CK >= ((int64_t)1 << 31)) return AS_ERR_LIMIT;
+  Plan pl;
+  e = make_plan(shape, tbar, layers, &pl);
+  if (e) return e;
+  if (grad_bytes) *grad_bytes = pl.total_grad;
+  return AS_OK;
+}
+
+size_t as_wcat_bytes(const as_shape_t* shape, int32_t layers) {
+  if (check_shape(shape) != AS_OK || layers < 1) return 0;
+  return (size_t)layers * (shape->d_model + NBC) * shape->d_model * (shape->io == AS_BF16 ? 2 : 4);
+}
+
+int as_pack_weights(const as_shape_t* shape, int32_t layers, const as_params_t* params, void* wcat, void* stream) {
+  int e = check_shape(shape);
+  if (e) return e;
+  e = check_params(params);
+  if (e) return e;
+  if (!wcat) return AS_ERR_NULL;
+  if (!aligned16(wcat)) return AS_ERR_ALIGN;
+  if (layers < 1) return AS_ERR_SHAPE;
+  if (shape->io != AS_BF16) return AS_ERR_DTYPE;   // only the bf16 tensor-core contractions read a packed copy
+  AS_TRY(tc_pack_wcat(shape->d_model, layers, params, wcat, reinterpret_cast<cudaStream_t>(stream)));
+  return AS_OK;
+}
+
+int as_adjoint_grad_layers(const as_shape_t* shape, int32_t layers, const as_params_t* params, const void* x,
+                           const void* dy, int64_t tbar, uint32_t flags, const as_grads_t* out, void* ws,
+                           size_t ws_bytes, void* stream) {
   int e = check_grad_args(shape, params, x, dy, out, ws);
   if (e) return e;
   if (tbar < 1) return AS_ERR_TBAR;
+  if (layers < 1) return AS_ERR_SHAPE;
+  if ((int64_t)layers * shape->batch * shape->seqlen + shape->seqlen + 2 * CK >= ((int64_t)1 << 31)) return AS_ERR_LIMIT;
   Plan pl;
-  e = make_plan(shape, tbar, &pl);
+  e = make_plan(shape, tbar, layers, &pl);
   if (e) return e;
   if (ws_bytes < pl.total_grad) return AS_ERR_WORKSPACE;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
@@ -247,7 +307,9 @@ int as_adjoint_grad(const as_shape_t* shape, const as_params_t* params, const vo
   mark(0, st);
   e = zero_outputs(pl, flags, out, w, st);
   if (e) return e;
-  e = projections(pl, params, x, w, st);
+  const void* wcat = nullptr;
+  if (pl.tc) { e = wcat_of(pl, params, w, st, &wcat); if (e) return e; }
+  e = projections(pl, params, wcat, x, w, st);
   if (e) return e;
   mark(1, st);
   ScanPtrs sp{x, dy, params->A_log, w};
@@ -257,7 +319,7 @@ int as_adjoint_grad(const as_shape_t* shape, const as_params_t* params, const vo
   mark(3, st);
   AS_TRY(launch_adjoint_main(pl, sp, out->dA_log, out->db_delta, st));
   mark(4, st);
-  e = contractions(pl, params, x, out, w, st);
+  e = contractions(pl, params, wcat, x, out, w, st);
   if (g_timing && e == AS_OK) g_timing_valid = true;
   return e;
 }
@@ -267,18 +329,20 @@ int as_full_bptt_grad(const as_shape_t* shape, const as_params_t* params, const 
   int e = check_grad_args(shape, params, x, dy, out, ws);
   if (e) return e;
   Plan pl;
-  e = make_plan(shape, shape->seqlen, &pl);
+  e = make_plan(shape, shape->seqlen, 1, &pl);
   if (e) return e;
   if (ws_bytes < pl.total_grad) return AS_ERR_WORKSPACE;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   char* w = reinterpret_cast<char*>(ws);
   e = zero_outputs(pl, flags, out, w, st);
   if (e) return e;
-  e = projections(pl, params, x, w, st);
+  const void* wcat = nullptr;
+  if (pl.tc) { e = wcat_of(pl, params, w, st, &wcat); if (e) return e; }
+  e = projections(pl, params, wcat, x, w, st);
   if (e) return e;
   ScanPtrs sp{x, dy, params->A_log, w};
   AS_TRY(launch_bptt(pl, sp, out->dA_log, out->db_delta, st));
-  return contractions(pl, params, x, out, w, st);
+  return contractions(pl, params, wcat, x, out, w, st);
 }
 
 int as_rmsnorm_fwd(const as_shape_t* shape, const void* y, void* yhat, float eps, void* stream) {

@@ -34,12 +34,14 @@ enum { MAJ_K = 0, MAJ_MN = 1 };
 enum { TC_PROJ = 0, TC_DW = 1, TC_DX = 2 };
 
 struct TcArgs {
-  int64_t M;            // rows of the output tile space (A's MN extent)
+  int64_t M;            // rows of the output tile space (A's MN extent); PROJ / DX: the tokens of all layers
   int N;                // cols of the output (B's MN extent)
-  int kblocks;          // number of BK-blocks along K
+  int kblocks;          // number of BK-blocks along K (DW: per layer)
   int splitk;
   int P;                // d_model
-  const float* bias;    // PROJ: b_delta
+  int layers;           // independent problems stacked along the leading dimension of every tensor
+  int64_t rows_layer;   // token rows per layer (a multiple of BM when layers > 1)
+  const float* bias;    // PROJ: b_delta [layers, P]
   int* status;
 };
 
@@ -157,7 +159,8 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 //   warps 2..9       : epilogue (two warps per TMEM lane quarter, each taking half of the columns); they drain
 //                      buffer a while the issuer already fills buffer a^1 for the next tile
 // Tile order: n fastest, then m, then the K split, so concurrently running CTAs share A rows through L2.
-template <int AMAJ, int BMAJ, int EPI, int BN>
+// ML: several layers stacked along the leading dimension of every tensor (false compiles the single-layer code).
+template <int AMAJ, int BMAJ, int EPI, int BN, bool ML>
 __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
                                                            const __grid_constant__ CUtensorMap tmB,
                                                            const __grid_constant__ CUtensorMap tmO0,
@@ -176,8 +179,9 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int mt = (int)((a.M + BM - 1) / BM), nt = (a.N + BN - 1) / BN;
-  const int ntiles = mt * nt * a.splitk;
+  const int ntiles = mt * nt * a.splitk * ((ML && EPI == TC_DW) ? a.layers : 1);
   const int kper = (a.kblocks + a.splitk - 1) / a.splitk;
+  const int NWc = a.P + NBC;                       // rows of one layer's Wcat
   volatile int* abortp = &abort_s;
 
   if (threadIdx.x == 0) {
@@ -197,9 +201,17 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = tmem_base_s;
 
-  auto decode = [&](int t, int64_t& m0, int& n0, int& kb0, int& nkb) {
-    const int in = t % nt, im = (t / nt) % mt, ik = t / (nt * mt);
+  // lay: the layer a tile belongs to.  PROJ / DX tile the token rows of all layers (a tile never straddles two layers);
+  // DW has its own set of (m, n, split) tiles per layer and contracts over that layer's tokens only.
+  auto decode = [&](int t, int64_t& m0, int& n0, int& kb0, int& nkb, int& lay) {
+    const int in = t % nt, im = (t / nt) % mt;
+    int ik = t / (nt * mt);
     m0 = (int64_t)im * BM; n0 = in * BN;
+    lay = 0;
+    if (ML) {
+      if (EPI == TC_DW) { lay = ik / a.splitk; ik -= lay * a.splitk; }
+      else lay = im / (int)(a.rows_layer / BM);
+    }
     kb0 = ik * kper;
     nkb = max(0, min(a.kblocks, kb0 + kper) - kb0);
   };
@@ -212,8 +224,11 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
       int it = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
-        int64_t m0; int n0, kb0, nkb;
-        decode(t, m0, n0, kb0, nkb);
+        int64_t m0; int n0, kb0, nkb, lay;
+        decode(t, m0, n0, kb0, nkb, lay);
+        // row offsets of this layer: DW contracts over its token rows (both operands), PROJ / DX read its Wcat rows
+        const int ktok = (ML && EPI == TC_DW) ? (int)(lay * a.rows_layer) : 0;
+        const int wrow = (ML && EPI != TC_DW) ? lay * NWc : 0;
         for (int i = 0; i < nkb; ++i, ++it) {
           const int s = it % STAGES, round = it / STAGES;
           if (round > 0 && !mbar_wait(&empty_bar[s], (round - 1) & 1, abortp)) { ok = false; break; }
@@ -224,14 +239,15 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
           if (AMAJ == MAJ_K) {
             tma_load_2d(sa, &tmA, k, (int)m0, &full_bar[s]);
           } else {
-            tma_load_2d(sa, &tmA, (int)m0, k, &full_bar[s]);
-            tma_load_2d(sa + A_BYTES / 2, &tmA, (int)m0 + 64, k, &full_bar[s]);
+            tma_load_2d(sa, &tmA, (int)m0, ktok + k, &full_bar[s]);
+            tma_load_2d(sa + A_BYTES / 2, &tmA, (int)m0 + 64, ktok + k, &full_bar[s]);
           }
           if (BMAJ == MAJ_K) {
-            tma_load_2d(sb, &tmB, k, n0, &full_bar[s]);
+            tma_load_2d(sb, &tmB, k, wrow + n0, &full_bar[s]);
           } else {
 #pragma unroll
-            for (int q = 0; q < BN / 64; ++q) tma_load_2d(sb + q * (64 * BK * 2), &tmB, n0 + 64 * q, k, &full_bar[s]);
+            for (int q = 0; q < BN / 64; ++q)
+              tma_load_2d(sb + q * (64 * BK * 2), &tmB, n0 + 64 * q, ktok + wrow + k, &full_bar[s]);
           }
         }
       }
@@ -245,8 +261,8 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
       int it = 0, ti = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++ti) {
-        int64_t m0; int n0, kb0, nkb;
-        decode(t, m0, n0, kb0, nkb);
+        int64_t m0; int n0, kb0, nkb, lay;
+        decode(t, m0, n0, kb0, nkb, lay);
         const int ab = ti & 1, around = ti >> 1;
         if (around > 0 && !mbar_wait(&tmem_empty_bar[ab], (around - 1) & 1, abortp)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -293,11 +309,12 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
     uint32_t nchunks_done = 0;                 // chunks this warp has staged so far (selects buffer and mbarrier phase)
     bool ok = true;
     for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++ti) {
-      int64_t m0; int n0, kb0, nkb;
-      decode(t, m0, n0, kb0, nkb);
+      int64_t m0; int n0, kb0, nkb, lay;
+      decode(t, m0, n0, kb0, nkb, lay);
       const int ab = ti & 1, around = ti >> 1;
       if (nkb > 0) {
         const int mrow = (int)m0 + quarter * 32;      // first output row of this warp
+        const float* bias_l = a.bias + (ML ? (int64_t)lay * a.P : 0);
         if (EPI == TC_DX && lane == 0 && n0 + c_lo * CW < a.N) {
           // dx_dir tile of the first chunk; later ones are requested one chunk ahead
           bulk_wait_read<0>();
@@ -348,7 +365,7 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
             if (lane == 0) bulk_wait_read<1>();         // the operation that last used this buffer has read it
             __syncwarp();
             if (EPI == TC_PROJ && nb < a.P) {
-              const float4* b4 = reinterpret_cast<const float4*>(a.bias + nb);
+              const float4* b4 = reinterpret_cast<const float4*>(bias_l + nb);
 #pragma unroll
               for (int q = 0; q < 4; ++q) {
                 const float4 bv = __ldg(b4 + q);
@@ -373,9 +390,10 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
                 for (int hh = 0; hh < 2; ++hh) {
                   const int mr = mrow + 16 * hh;
                   const void* src = buf + hh * 1024;
-                  if (mr < a.P) tma_reduce_add_2d(&tmO0, src, nb, mr);
-                  else if (mr < a.P + NS) tma_reduce_add_2d(&tmO1, src, nb, mr - a.P);
-                  else if (mr < a.P + 2 * NS) tma_reduce_add_2d(&tmO2, src, nb, mr - a.P - NS);
+                  const int l1 = ML ? lay * a.P : 0, l2 = ML ? lay * NS : 0;   // this layer's rows of the stacked outputs
+                  if (mr < a.P) tma_reduce_add_2d(&tmO0, src, nb, l1 + mr);
+                  else if (mr < a.P + NS) tma_reduce_add_2d(&tmO1, src, nb, l2 + mr - a.P);
+                  else if (mr < a.P + 2 * NS) tma_reduce_add_2d(&tmO2, src, nb, l2 + mr - a.P - NS);
                 }
               }
               bulk_commit();
@@ -401,11 +419,14 @@ __global__ void __launch_bounds__(NTHREADS) gemm_tc_kernel(const __grid_constant
 }
 
 // ---- small helpers -------------------------------------------------------------------------------
+// Wcat[l] = [W_delta[l]; W_B[l]; W_C[l]] for every layer l (blockIdx.y)
 __global__ void pack_wcat_kernel(int P, const __nv_bfloat16* __restrict__ Wd, const __nv_bfloat16* __restrict__ WB,
                                  const __nv_bfloat16* __restrict__ WC, __nv_bfloat16* __restrict__ out) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int64_t n = (int64_t)(P + NBC) * P;
   if (i >= n) return;
+  const int64_t l = blockIdx.y;
+  Wd += l * P * P; WB += l * NS * P; WC += l * NS * P; out += l * n;
   const int64_t row = i / P, col = i % P;
   out[i] = row < P ? Wd[i] : (row < P + NS ? WB[(row - P) * P + col] : WC[(row - P - NS) * P + col]);
 }
@@ -467,12 +488,12 @@ int make_map_out_bf16(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t
   return make_map_t(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, CU_TENSOR_MAP_SWIZZLE_64B, base, rows, cols, cols, 32, 32);
 }
 
-template <int AMAJ, int BMAJ, int EPI, int BN>
-int launch_tc(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap (&tmO)[3], const TcArgs& a, cudaStream_t st) {
-  auto kern = gemm_tc_kernel<AMAJ, BMAJ, EPI, BN>;
+template <int AMAJ, int BMAJ, int EPI, int BN, bool ML>
+int launch_tc_ml(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap (&tmO)[3], const TcArgs& a, cudaStream_t st) {
+  auto kern = gemm_tc_kernel<AMAJ, BMAJ, EPI, BN, ML>;
   static bool done[AS_MAX_DEVICES] = {};
   if (ensure_dynamic_smem(kern, Cfg<BN>::SMEM_DYN, done)) return 1;
-  const int64_t ntiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN) * a.splitk;
+  const int64_t ntiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN) * a.splitk * (EPI == TC_DW ? a.layers : 1);
   const int sms = sm_count();
   const unsigned grid = (unsigned)(ntiles < sms ? ntiles : sms);   // one persistent CTA per SM
   kern<<<grid, NTHREADS, Cfg<BN>::SMEM_DYN, st>>>(tmA, tmB, tmO[0], tmO[1], tmO[2], a);
@@ -480,77 +501,116 @@ int launch_tc(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap 
   return (int)cudaGetLastError();
 }
 
+template <int AMAJ, int BMAJ, int EPI, int BN>
+int launch_tc(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap (&tmO)[3], const TcArgs& a, cudaStream_t st) {
+  return a.layers > 1 ? launch_tc_ml<AMAJ, BMAJ, EPI, BN, true>(tmA, tmB, tmO, a, st)
+                      : launch_tc_ml<AMAJ, BMAJ, EPI, BN, false>(tmA, tmB, tmO, a, st);
+}
+
 }  // namespace
 
 constexpr int TBN = 256;   // tile width of the weight-gradient and input-gradient contractions
 constexpr int PBN = 208;   // projections: N = P + 32; for P = 768 four 208-wide tiles waste 4 % where 256 wastes 22 %
 
-int tc_pack_wcat(const Plan& pl, const as_params_t* pr, char* ws, cudaStream_t st) {
-  const int64_t n = (int64_t)(pl.P + NBC) * pl.P;
-  pack_wcat_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(
-      pl.P, (const __nv_bfloat16*)pr->W_delta, (const __nv_bfloat16*)pr->W_B, (const __nv_bfloat16*)pr->W_C,
-      (__nv_bfloat16*)(ws + pl.off_wcat));
+int tc_pack_wcat(int P, int layers, const as_params_t* pr, void* wcat, cudaStream_t st) {
+  const int64_t n = (int64_t)(P + NBC) * P;
+  pack_wcat_kernel<<<dim3((unsigned)((n + 255) / 256), (unsigned)layers), 256, 0, st>>>(
+      P, (const __nv_bfloat16*)pr->W_delta, (const __nv_bfloat16*)pr->W_B, (const __nv_bfloat16*)pr->W_C,
+      (__nv_bfloat16*)wcat);
   count_launch();
   return (int)cudaGetLastError();
 }
 
-int tc_projections(const Plan& pl, const as_params_t* pr, const void* x, char* ws, cudaStream_t st) {
-  const int64_t M = (int64_t)pl.B * pl.T;
+// The layers of a call go out as one launch when no 128-row tile straddles two layers (token rows per layer a
+// multiple of BM); otherwise one launch per layer, on that layer's slab of every tensor.
+struct LayerLoop { int first, count; };
+static inline int layer_groups(const Plan& pl, LayerLoop* g) {
+  const int64_t rows = (int64_t)pl.Bg * pl.T;
+  if (pl.KL == 1 || rows % BM == 0) { g[0] = {0, pl.KL}; return 1; }
+  return 0;   // the caller loops over single layers
+}
+
+int tc_projections(const Plan& pl, const as_params_t* pr, const void* wcat, const void* x, char* ws, cudaStream_t st) {
+  const int64_t rows = (int64_t)pl.Bg * pl.T;
   const int P = pl.P, NW = P + NBC;
-  CUtensorMap tmA, tmB;
-  if (make_map(&tmA, x, M, P, P, BM)) return 1;
-  if (make_map(&tmB, ws + pl.off_wcat, NW, P, P, PBN)) return 1;
-  TcArgs a{};
-  a.M = M; a.N = NW; a.kblocks = (P + BK - 1) / BK; a.splitk = 1; a.P = P;
-  a.bias = pr->b_delta;
-  a.status = (int*)(ws + pl.off_status);
-  CUtensorMap tmO[3];
-  if (make_map_out_f32(&tmO[0], ws + pl.off_delta, M, P, 32)) return 1;
-  if (make_map_out_f32(&tmO[1], ws + pl.off_bc, M, NBC, 32)) return 1;
-  tmO[2] = tmO[1];
-  return launch_tc<MAJ_K, MAJ_K, TC_PROJ, PBN>(tmA, tmB, tmO, a, st);
+  LayerLoop one;
+  const bool batched = layer_groups(pl, &one) == 1;
+  for (int l0 = 0; l0 < pl.KL; l0 += batched ? pl.KL : 1) {
+    const int nl = batched ? pl.KL : 1;
+    const int64_t M = rows * nl;
+    CUtensorMap tmA, tmB;
+    if (make_map(&tmA, (const char*)x + (size_t)l0 * rows * P * 2, M, P, P, BM)) return 1;
+    if (make_map(&tmB, (const char*)wcat + (size_t)l0 * NW * P * 2, (uint64_t)NW * nl, P, P, PBN)) return 1;
+    TcArgs a{};
+    a.M = M; a.N = NW; a.kblocks = (P + BK - 1) / BK; a.splitk = 1; a.P = P; a.layers = nl; a.rows_layer = rows;
+    a.bias = pr->b_delta + (size_t)l0 * P;
+    a.status = (int*)(ws + pl.off_status);
+    CUtensorMap tmO[3];
+    if (make_map_out_f32(&tmO[0], ws + pl.off_delta + (size_t)l0 * rows * P * 4, M, P, 32)) return 1;
+    if (make_map_out_f32(&tmO[1], ws + pl.off_bc + (size_t)l0 * rows * NBC * 4, M, NBC, 32)) return 1;
+    tmO[2] = tmO[1];
+    const int e = launch_tc<MAJ_K, MAJ_K, TC_PROJ, PBN>(tmA, tmB, tmO, a, st);
+    if (e) return e;
+  }
+  return 0;
 }
 
 int tc_weight_grads(const Plan& pl, const void* x, const as_grads_t* out, char* ws, cudaStream_t st) {
-  const int64_t M = (int64_t)pl.B * pl.T;
+  const int64_t rows = (int64_t)pl.Bg * pl.T;
+  const int64_t Mall = rows * pl.KL;
   const int P = pl.P, NW = P + NBC;
-  cvt_dbc_kernel<<<(unsigned)((M * (NBC / 8) + 255) / 256), 256, 0, st>>>(M, NW, P, (const float*)(ws + pl.off_dbc),
-                                                                    (__nv_bfloat16*)(ws + pl.off_du));
+  cvt_dbc_kernel<<<(unsigned)((Mall * (NBC / 8) + 255) / 256), 256, 0, st>>>(Mall, NW, P, (const float*)(ws + pl.off_dbc),
+                                                                       (__nv_bfloat16*)(ws + pl.off_du));
   count_launch();
   if (cudaGetLastError() != cudaSuccess) return 1;
-  CUtensorMap tmA, tmB;
-  if (make_map(&tmA, ws + pl.off_du, M, NW, NW, 64)) return 1;   // Gcat as [K=tokens, M=P+32]
-  if (make_map(&tmB, x, M, P, P, 64)) return 1;                  // X as [K=tokens, N=P]
-  TcArgs a{};
-  a.M = NW; a.N = P; a.kblocks = (int)((M + BK - 1) / BK); a.P = P;
-  const int tiles = ((NW + BM - 1) / BM) * ((P + TBN - 1) / TBN);
-  int sk = (sm_count() * 2) / tiles;   // about two tiles per persistent CTA
-  if (sk > a.kblocks) sk = a.kblocks;
-  if (sk < 1) sk = 1;
-  const int kper = (a.kblocks + sk - 1) / sk;
-  a.splitk = (a.kblocks + kper - 1) / kper;   // no empty split: every tile has at least one K block
-  a.status = (int*)(ws + pl.off_status);
-  CUtensorMap tmO[3];
-  if (make_map_out_f32(&tmO[0], out->dW_delta, P, P, 16)) return 1;
-  if (make_map_out_f32(&tmO[1], out->dW_B, NS, P, 16)) return 1;
-  if (make_map_out_f32(&tmO[2], out->dW_C, NS, P, 16)) return 1;
-  return launch_tc<MAJ_MN, MAJ_MN, TC_DW, TBN>(tmA, tmB, tmO, a, st);
+  LayerLoop one;
+  const bool batched = layer_groups(pl, &one) == 1;
+  for (int l0 = 0; l0 < pl.KL; l0 += batched ? pl.KL : 1) {
+    const int nl = batched ? pl.KL : 1;
+    CUtensorMap tmA, tmB;
+    if (make_map(&tmA, ws + pl.off_du + (size_t)l0 * rows * NW * 2, rows * nl, NW, NW, 64)) return 1;   // Gcat as [K=tokens, M=P+32]
+    if (make_map(&tmB, (const char*)x + (size_t)l0 * rows * P * 2, rows * nl, P, P, 64)) return 1;       // X as [K=tokens, N=P]
+    TcArgs a{};
+    a.M = NW; a.N = P; a.kblocks = (int)((rows + BK - 1) / BK); a.P = P; a.layers = nl; a.rows_layer = rows;
+    const int tiles = ((NW + BM - 1) / BM) * ((P + TBN - 1) / TBN) * nl;
+    int sk = (sm_count() * 2) / tiles;   // about two tiles per persistent CTA
+    if (sk > a.kblocks) sk = a.kblocks;
+    if (sk < 1) sk = 1;
+    const int kper = (a.kblocks + sk - 1) / sk;
+    a.splitk = (a.kblocks + kper - 1) / kper;   // no empty split: every tile has at least one K block
+    a.status = (int*)(ws + pl.off_status);
+    CUtensorMap tmO[3];
+    if (make_map_out_f32(&tmO[0], out->dW_delta + (size_t)l0 * P * P, (uint64_t)P * nl, P, 16)) return 1;
+    if (make_map_out_f32(&tmO[1], out->dW_B + (size_t)l0 * NS * P, (uint64_t)NS * nl, P, 16)) return 1;
+    if (make_map_out_f32(&tmO[2], out->dW_C + (size_t)l0 * NS * P, (uint64_t)NS * nl, P, 16)) return 1;
+    const int e = launch_tc<MAJ_MN, MAJ_MN, TC_DW, TBN>(tmA, tmB, tmO, a, st);
+    if (e) return e;
+  }
+  return 0;
 }
 
-int tc_input_grad(const Plan& pl, void* dx, char* ws, cudaStream_t st) {
-  const int64_t M = (int64_t)pl.B * pl.T;
+int tc_input_grad(const Plan& pl, const void* wcat, void* dx, char* ws, cudaStream_t st) {
+  const int64_t rows = (int64_t)pl.Bg * pl.T;
   const int P = pl.P, NW = P + NBC;
-  CUtensorMap tmA, tmB;
-  if (make_map(&tmA, ws + pl.off_du, M, NW, NW, BM)) return 1;       // Gcat as [M=tokens, K=P+32]
-  if (make_map(&tmB, ws + pl.off_wcat, NW, P, P, 64)) return 1;      // Wcat as [K=P+32, N=P]
-  TcArgs a{};
-  a.M = M; a.N = P; a.kblocks = (NW + BK - 1) / BK; a.splitk = 1; a.P = P;
-  a.status = (int*)(ws + pl.off_status);
-  CUtensorMap tmO[3];
-  if (make_map_out_bf16(&tmO[0], dx, M, P)) return 1;
-  if (make_map_out_bf16(&tmO[1], ws + pl.off_dxdir, M, P)) return 1;
-  tmO[2] = tmO[1];
-  return launch_tc<MAJ_K, MAJ_MN, TC_DX, TBN>(tmA, tmB, tmO, a, st);
+  LayerLoop one;
+  const bool batched = layer_groups(pl, &one) == 1;
+  for (int l0 = 0; l0 < pl.KL; l0 += batched ? pl.KL : 1) {
+    const int nl = batched ? pl.KL : 1;
+    const int64_t M = rows * nl;
+    CUtensorMap tmA, tmB;
+    if (make_map(&tmA, ws + pl.off_du + (size_t)l0 * rows * NW * 2, M, NW, NW, BM)) return 1;            // Gcat as [M=tokens, K=P+32]
+    if (make_map(&tmB, (const char*)wcat + (size_t)l0 * NW * P * 2, (uint64_t)NW * nl, P, P, 64)) return 1;   // Wcat as [K=P+32, N=P]
+    TcArgs a{};
+    a.M = M; a.N = P; a.kblocks = (NW + BK - 1) / BK; a.splitk = 1; a.P = P; a.layers = nl; a.rows_layer = rows;
+    a.status = (int*)(ws + pl.off_status);
+    CUtensorMap tmO[3];
+    if (make_map_out_bf16(&tmO[0], (char*)dx + (size_t)l0 * rows * P * 2, M, P)) return 1;
+    if (make_map_out_bf16(&tmO[1], ws + pl.off_dxdir + (size_t)l0 * rows * P * 2, M, P)) return 1;
+    tmO[2] = tmO[1];
+    const int e = launch_tc<MAJ_K, MAJ_MN, TC_DX, TBN>(tmA, tmB, tmO, a, st);
+    if (e) return e;
+  }
+  return 0;
 }
 
 }  // namespace as

@@ -79,7 +79,9 @@ __device__ __forceinline__ float ex2_approx(float x) {
 // (float4 q of thread tid at float offset (q*NTHR + tid)*4), so one bulk copy moves a CTA's block and
 // every thread's access is a contiguous 16 bytes.
 struct Plan {
-  int B, P;
+  int KL;           // layers handled by one call (independent problems that share dy); 1 for the single-layer entry points
+  int Bg;           // batch elements per layer
+  int B, P;         // B = KL * Bg: the kernels see (layer, batch element) as one batch index; layer = b / Bg
   int64_t T;
   int64_t tbar;     // clamped to T
   int full;         // tbar >= T
@@ -100,7 +102,9 @@ struct Plan {
       off_bptt_ckpt, off_wcat, total_fwd, total_grad;
 };
 
-int make_plan(const as_shape_t* sh, int64_t tbar, Plan* pl);
+int make_plan(const as_shape_t* sh, int64_t tbar, int layers, Plan* pl);
+// elements of A_log (and dA_log) per layer
+inline int64_t a_stride(const Plan& pl) { return pl.scalar ? (int64_t)pl.P : (int64_t)pl.P * NS; }
 
 // ---- launchers (each returns a cudaError_t as int) ------------------------------------------
 // C[m, coff + n] (ldc) = epi( sum_k A(m,k) B(n,k) ), fp32 accumulation on the FP32 pipe.
@@ -129,10 +133,10 @@ int launch_wait_selftest(int* status, unsigned limit, cudaStream_t st);
 int launch_finish_dx(const Plan& pl, const float* dxacc, const void* dxdir, void* dx, cudaStream_t st);
 
 // bf16 tensor-core path (as_gemm_tc.cu)
-int tc_pack_wcat(const Plan& pl, const as_params_t* pr, char* ws, cudaStream_t st);
-int tc_projections(const Plan& pl, const as_params_t* pr, const void* x, char* ws, cudaStream_t st);
+int tc_pack_wcat(int P, int layers, const as_params_t* pr, void* wcat, cudaStream_t st);
+int tc_projections(const Plan& pl, const as_params_t* pr, const void* wcat, const void* x, char* ws, cudaStream_t st);
 int tc_weight_grads(const Plan& pl, const void* x, const as_grads_t* out, char* ws, cudaStream_t st);
-int tc_input_grad(const Plan& pl, void* dx, char* ws, cudaStream_t st);
+int tc_input_grad(const Plan& pl, const void* wcat, void* dx, char* ws, cudaStream_t st);
 
 int launch_bptt(const Plan& pl, const ScanPtrs& sp, float* dA_log, float* db_delta, cudaStream_t st);
 

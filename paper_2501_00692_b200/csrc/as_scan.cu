@@ -14,6 +14,8 @@
 // instead of registers or shared memory.
 #include <cuda.h>
 
+#include <type_traits>
+
 #include "as_internal.cuh"
 
 namespace as {
@@ -23,9 +25,10 @@ namespace as {
 // ------------------------------------------------------------------------------------------------
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-int make_plan(const as_shape_t* sh, int64_t tbar, Plan* pl) {
+int make_plan(const as_shape_t* sh, int64_t tbar, int layers, Plan* pl) {
   Plan p{};
-  p.B = sh->batch; p.P = sh->d_model; p.T = sh->seqlen; p.io = sh->io;
+  p.KL = layers < 1 ? 1 : layers; p.Bg = sh->batch;
+  p.B = p.KL * p.Bg; p.P = sh->d_model; p.T = sh->seqlen; p.io = sh->io;
   p.scalar = sh->a_structure == AS_A_SCALAR ? 1 : 0;
   p.tc = (sh->io == AS_BF16 && sh->d_model % 32 == 0) ? 1 : 0;
   p.du_ld = p.tc ? p.P + NBC : p.P;
@@ -35,7 +38,7 @@ int make_plan(const as_shape_t* sh, int64_t tbar, Plan* pl) {
   p.bw = p.P < CH ? p.P : CH;
   const int64_t ctas = (int64_t)p.tiles * p.B;
   // two full waves of the main kernel's resident CTAs (148 SMs x CTAs per SM), never more than that
-  const int64_t slots = (int64_t)sm_count() * AS_MAIN_CTAS;
+  const int64_t slots = (int64_t)sm_count() * 3;   // resident CTAs of the main kernel
   int64_t s_target = (2 * slots) / ctas;
   if (s_target < 1) s_target = 1;
   int64_t L = (p.T + s_target - 1) / s_target;
@@ -60,7 +63,7 @@ int make_plan(const as_shape_t* sh, int64_t tbar, Plan* pl) {
   p.off_hend = take(BSB * 4);
   p.off_segd = take(BSP * 4);
   p.off_hstart = take(BSB * 4);
-  p.off_wcat = take((size_t)(p.P + NBC) * p.P * 2);
+  p.off_wcat = take((size_t)p.KL * (p.P + NBC) * p.P * 2);
   p.total_fwd = o;
   p.off_ckpt = take((size_t)p.B * p.NC * p.tiles * TILE_FLOATS * 4);
   p.off_cs = take((size_t)p.B * p.NC * p.P * 4);
@@ -76,12 +79,14 @@ int make_plan(const as_shape_t* sh, int64_t tbar, Plan* pl) {
   p.off_bptt_ckpt = take((size_t)p.B * ((p.T + 63) / 64) * p.P * NS * 4);
   p.total_grad = o;
   *pl = p;
-  return p.S > 65535 ? AS_ERR_LIMIT : AS_OK;   // segments fill gridDim.y
+  return (p.S > 65535 || p.B > 65535) ? AS_ERR_LIMIT : AS_OK;   // segments fill gridDim.y, (layer, batch) gridDim.z
 }
 
 namespace {
 
 typedef unsigned long long u64;   // two packed fp32 values (lo = even state, hi = odd state)
+
+__device__ __forceinline__ int64_t a_stride_dev(const Plan& pl) { return pl.scalar ? (int64_t)pl.P : (int64_t)pl.P * NS; }
 
 __device__ __forceinline__ u64 pk(float lo, float hi) {
   u64 r;
@@ -156,22 +161,9 @@ struct Stage {
 };
 constexpr int NSTAGE = 3;        // ascending kernels
 constexpr int WRED_Q = 32 * 4 + 8;   // floats per quarter-block of the per-warp reduction scratch (512 B + 32 B skew)
-#ifndef AS_MAIN_CTAS
-#define AS_MAIN_CTAS 3
-#endif
-#ifndef AS_PARK_ABAR
-#define AS_PARK_ABAR 0
-#endif
-constexpr int MAIN_CTAS = AS_MAIN_CTAS;    // resident CTAs per SM the main kernel is compiled for
-constexpr bool PARK_ABAR = AS_PARK_ABAR != 0;   // park abar_j next to h_j in tensor memory: the backward walk then needs no ex2
-#ifndef AS_FW_UNROLL
-#define AS_FW_UNROLL 4
-#endif
-#ifndef AS_BW_UNROLL
-#define AS_BW_UNROLL 2
-#endif
-constexpr int FW_UNROLL = AS_FW_UNROLL;     // unroll factor of the main adjoint kernel's forward rebuild loop
-constexpr int BW_UNROLL = AS_BW_UNROLL;     // unroll factor of the main adjoint kernel's backward token loop
+constexpr int MAIN_CTAS = 3;    // resident CTAs per SM the main kernel is compiled for (up to 168 registers per thread)
+constexpr int FW_UNROLL = 4;     // unroll factor of the main adjoint kernel's forward rebuild loop
+constexpr int BW_UNROLL = 2;     // unroll factor of the main adjoint kernel's backward token loop
 constexpr int NSTAGE_MAIN = 2;   // main adjoint kernel: a chunk takes thousands of cycles, one chunk of lookahead suffices
 
 // per-thread values of its NCH channels
@@ -326,6 +318,8 @@ __global__ void __launch_bounds__(NTHR, 4) ascend_kernel(const __grid_constant__
   const int nchunk = (int)((t1 - t0 + CK - 1) / CK);
   const float* bc = reinterpret_cast<const float*>(ws + pl.off_bc);
   int* status = reinterpret_cast<int*>(ws + pl.off_status);
+  A_log += (int64_t)(b / pl.Bg) * a_stride_dev(pl);   // this layer's rates
+  const int bg = b % pl.Bg;                            // dy is shared by the layers: its rows know only the batch element
 
   if (w.tid == 0) {
     for (int i = 0; i < NSTAGE; ++i) mbar_init(&full_bar[i], 1);
@@ -340,7 +334,7 @@ __global__ void __launch_bounds__(NTHR, 4) ascend_kernel(const __grid_constant__
     mbar_expect_tx(&full_bar[st], tx_bytes);
     tma_2d(sm + St::X, &tmX, tile * CH, row, &full_bar[st]);
     tma_2d(sm + St::D, &tmD, tile * CH, row, &full_bar[st]);
-    if (MU) tma_2d(sm + St::G, &tmG, tile * CH, row, &full_bar[st]);
+    if (MU) tma_2d(sm + St::G, &tmG, tile * CH, (int64_t)bg * pl.T + t0 + (int64_t)c * CK, &full_bar[st]);
     bulk_1d(sm + St::BC, bc + row * NBC, CK * NBC * 4, &full_bar[st]);
   };
   if (w.tid == 0)
@@ -493,6 +487,7 @@ __global__ void __launch_bounds__(NTHR, 4) ascend_kernel(const __grid_constant__
 __global__ void __launch_bounds__(NTHR) fixup_h_kernel(Plan pl, const float* __restrict__ A_log, char* __restrict__ ws) {
   const int tile = blockIdx.x, b = blockIdx.y, u = blockIdx.z;
   const Who w = who(tile, pl.P);
+  A_log += (int64_t)(b / pl.Bg) * a_stride_dev(pl);
   u64 A2all[NU];
   load_A2(A_log, w, A2all, pl.scalar);
   u64 A2u = 0ull;
@@ -548,6 +543,7 @@ __global__ void __launch_bounds__(NTHR) fixup_mu_kernel(Plan pl, const float* __
   const int tile = blockIdx.x, b = blockIdx.z;
   const int P = pl.P, S = pl.S;
   const Who w = who(tile, P);
+  A_log += (int64_t)(b / pl.Bg) * a_stride_dev(pl);
   u64 A2[NU];
   load_A2(A_log, w, A2, pl.scalar);
   const float* muloc = reinterpret_cast<const float*>(ws + pl.off_muloc);
@@ -630,8 +626,8 @@ __device__ __forceinline__ void decay_units(const u64 (&e2)[NCH], const u64 (&A2
 // columns of its SM (three CTAs are resident) and every thread parks the chunk's eight states in its own TMEM lane:
 // warp w of the 4-warp CTA owns lanes [32w, 32w+32), a 32x32b access moves 16 registers of each lane to or
 // from 16 consecutive columns.
-constexpr int TM_TOK = PARK_ABAR ? 32 : 16;   // columns per token: h_j (16) and, when parked, abar_j (16)
-constexpr int TM_COLS = CK * TM_TOK;
+constexpr int TM_TOK = 16;         // columns per token: the 16 state registers of a thread
+constexpr int TM_COLS = CK * TM_TOK;   // columns [16 j, 16 j + 16): state after token j of the current chunk
 
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const u64 (&v)[NU]) {
   uint32_t r[16];
@@ -655,28 +651,6 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, u64 (&v)[NU]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
   for (int u = 0; u < 8; ++u) asm("mov.b64 %0, {%1, %2};" : "=l"(v[u]) : "r"(r[2 * u]), "r"(r[2 * u + 1]));
-}
-// two 16-column loads behind one wait
-__device__ __forceinline__ void tmem_ld16x2(uint32_t taddr, u64 (&v)[NU], u64 (&w2)[NU]) {
-  uint32_t r[16], q[16];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(q[0]), "=r"(q[1]), "=r"(q[2]), "=r"(q[3]), "=r"(q[4]), "=r"(q[5]), "=r"(q[6]), "=r"(q[7]), "=r"(q[8]),
-        "=r"(q[9]), "=r"(q[10]), "=r"(q[11]), "=r"(q[12]), "=r"(q[13]), "=r"(q[14]), "=r"(q[15])
-      : "r"(taddr + 16)
-      : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int u = 0; u < 8; ++u) {
-    asm("mov.b64 %0, {%1, %2};" : "=l"(v[u]) : "r"(r[2 * u]), "r"(r[2 * u + 1]));
-    asm("mov.b64 %0, {%1, %2};" : "=l"(w2[u]) : "r"(q[2 * u]), "r"(q[2 * u + 1]));
-  }
 }
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -740,6 +714,13 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   int* status = reinterpret_cast<int*>(ws + pl.off_status);
   const int ncs = min(CH, P - tile * CH);   // channels of this tile that exist
   const int64_t BT = (int64_t)pl.B * T;
+  {   // this layer's rates and parameter-gradient rows; dy is shared by the layers
+    const int lay = b / pl.Bg;
+    A_log += (int64_t)lay * a_stride_dev(pl);
+    dA_log += (int64_t)lay * a_stride_dev(pl);
+    db_delta += (int64_t)lay * P;
+  }
+  const int64_t grow0 = (int64_t)(b % pl.Bg) * T - (int64_t)b * T;   // added to an x / Delta row to get the dy row
   const int du_ld = pl.du_ld;
   // the two lanes of a pair end up with the same per-channel sums: lane `half` finalises channel `half`
   const int chf = w.half;
@@ -767,8 +748,43 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tm = tmem_base_s + ((uint32_t)(32 * warp) << 16);   // this warp's lanes, column 0 of the allocation
+  // Window liveness of the whole segment, decided before anything is loaded for it.  For every token i of segment s
+  // the window (i, i + Tbar] contains the m - 1 whole segments s+1 .. s+m-1 (m = Tbar / L), so the sum of their Delta
+  // is a lower bound of every window sum of the segment.  If that bound already gives an exit factor below 2^-64 for
+  // every state of every channel of the tile, no exit term of the segment can matter (far below one rounding unit of
+  // mu): the rows Tbar ahead are then neither loaded nor looked at.
+  bool seg_dead = false;
+  if (WIN) {
+    float lb[NCH];
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) lb[c] = 0.f;
+    if (w.act) {
+      const float* segd = reinterpret_cast<const float*>(ws + pl.off_segd);
+      for (int k2 = 1; k2 < pl.m && s + k2 < pl.S; ++k2) {
+        const ChV v = ldg_ch(segd + ((int64_t)b * pl.S + s + k2) * P + w.pa);
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) lb[c] += v.v[c];
+      }
+    }
+    bool dead = true;   // channels that do not exist never veto
+    if (w.act) {
+      // least negative exponent scale of each channel over this thread's 8 states; the pair lane tests its own 8
+      const float* al = A_log + (pl.scalar ? (int64_t)w.pa : (int64_t)w.pa * NS + 8 * w.half);
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) {
+        float mn = 3.0e38f;   // smallest A_log = least negative A
+        if (pl.scalar) mn = __ldg(al + c);
+        else
+          for (int n = 0; n < 8; ++n) mn = fminf(mn, __ldg(al + c * NS + n));
+        dead = dead && (lb[c] * (-__expf(mn) * LOG2E) <= -64.f);
+      }
+      // a window that reaches past the sequence end has no exit term at all; tokens whose window ends inside it do
+    }
+    seg_dead = __syncthreads_and(dead ? 1 : 0) != 0;
+  }
+  const bool win_on = WIN && !seg_dead;
   const uint32_t tx_base = (uint32_t)(CK * CH * ESZ * 2 + CK * CH * 4 + CK * NBC * 4 + ncs * 4 +
-                                      (WIN ? CK * CH * ESZ + CK * CH * 4 : 0));
+                                      (win_on ? CK * CH * ESZ + CK * CH * 4 : 0));
   // chunks are visited last to first: the i-th visited chunk is c = nchunk-1-i
   auto issue = [&](int i) {
     const int st = i % NSTAGE_MAIN;
@@ -778,17 +794,17 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     const int64_t row = (int64_t)b * T + tc;
     const int64_t cc = (int64_t)b * pl.NC + tc / CK;
     const int64_t row2 = row + tbar;             // first token leaving the window of this chunk's tokens
-    const bool win_rows = WIN && row2 < BT;      // its B/C rows exist (else no token of the chunk has t + Tbar < T)
+    const bool win_rows = win_on && row2 < BT;   // its B/C rows exist (else no token of the chunk has t + Tbar < T)
     mbar_expect_tx(&full_bar[st], tx_base + (win_rows ? CK * NBC * 4 : 0));
     tma_2d(sm + St::X, &tmX, tile * CH, row, &full_bar[st]);
     tma_2d(sm + St::D, &tmD, tile * CH, row, &full_bar[st]);
-    tma_2d(sm + St::G, &tmG, tile * CH, row, &full_bar[st]);
+    tma_2d(sm + St::G, &tmG, tile * CH, row + grow0, &full_bar[st]);
     bulk_1d(sm + St::BC, bc + row * NBC, CK * NBC * 4, &full_bar[st]);
     bulk_1d(sm + St::CS, cs + cc * P + tile * CH, ncs * 4, &full_bar[st]);
-    if (WIN) {
+    if (win_on) {
       // rows of the tokens leaving the window; past the end of the whole tensor TMA fills zeros, and rows
       // that belong to the next batch element are masked out below (t + Tbar < T fails)
-      tma_2d(sm + St::G2, &tmG, tile * CH, row2, &full_bar[st]);
+      tma_2d(sm + St::G2, &tmG, tile * CH, row2 + grow0, &full_bar[st]);
       tma_2d(sm + St::D2, &tmD, tile * CH, row2, &full_bar[st]);
       if (win_rows) bulk_1d(sm + St::BC2, bc + row2 * NBC, CK * NBC * 4, &full_bar[st]);
     }
@@ -828,7 +844,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   double sw[NCH];
 #pragma unroll
   for (int c = 0; c < NCH; ++c) sw[c] = 0.0;
-  if (WIN && w.act) {
+  if (win_on && w.act) {
     const double* swp = reinterpret_cast<const double*>(ws + pl.off_swin) + ((int64_t)b * pl.S + s) * P + w.pa;
 #pragma unroll
     for (int c = 0; c < NCH; ++c) sw[c] = swp[c];
@@ -837,6 +853,10 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   bool failed = false;
   int fail_i = 0, ckp_issued = 0;   // thread 0: where the walk stopped, last checkpoint copy issued
 
+  // The walk over the segment's chunks, compiled twice: with the window-exit terms and without them (the full form,
+  // and every segment whose exit terms were ruled out above).
+  auto walk_segment = [&](auto winon_tag) {
+  constexpr bool WINON = decltype(winon_tag)::value;
   for (int i = 0; i < nchunk; ++i) {
     const int st = i % NSTAGE_MAIN;
     const int c = nchunk - 1 - i;
@@ -847,7 +867,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     const int64_t tc = t0 + (int64_t)c * CK;
     const int nt = (int)min((int64_t)CK, t1 - tc);
     const int rb = i & 1;
-    const int nwin = WIN ? (int)max((int64_t)0, min((int64_t)CK, T - tbar - tc)) : 0;   // tokens j < nwin have t + Tbar < T
+    const int nwin = WINON ? (int)max((int64_t)0, min((int64_t)CK, T - tbar - tc)) : 0;   // tokens j < nwin have t + Tbar < T
     // window Delta sum: fp64 value at the chunk's last token + an fp32 running offset inside the chunk
     float swc[NCH], swl[NCH], dsumc[NCH], sd2[NCH];
 #pragma unroll
@@ -885,7 +905,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
 #pragma unroll
         for (int u = 0; u < NU; ++u) h[u] = fma2(dec[u], hst[u], h[u]);
       }
-      if (WIN) {
+      if (WINON) {
         // Delta of the tokens leaving the window during this chunk.  Inside the chunk the window sum never drops
         // below (sum at the chunk's last token) - (their total), so if even that bound gives W < 2^-64 for every
         // state of every lane, the exit terms of the whole chunk are skipped: they are far below one rounding unit
@@ -923,7 +943,6 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
 #pragma unroll
           for (int u = 0; u < NU; ++u) h[u] = fma2(af[u], h[u], mul2(dx2[u / 4], Bp[u % 4]));
           tmem_st16(tm + TM_TOK * j, h);
-          if (PARK_ABAR) tmem_st16(tm + TM_TOK * j + 16, af);
         }
         tmem_wait_st();
       }
@@ -944,9 +963,8 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
       uint32_t tmj = tm + TM_TOK * (CK - 1);
 #pragma unroll BW_UNROLL
       for (int j = CK - 1; j >= 0; --j) {
-        u64 hT[NU], aT[NU];
-        if (PARK_ABAR) tmem_ld16x2(tmj, hT, aT);
-        else tmem_ld16(tmj, hT);
+        u64 hT[NU];
+        tmem_ld16(tmj, hT);
         tmj -= TM_TOK;
         const ChV dv = lds_chp<float>(pD);
         const ChV xv = lds_chp<IO>(pX);
@@ -970,7 +988,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         for (int u = 0; u < NU; ++u) mu[u] = fma2(g2[u / 4], Cp[u % 4], mu[u]);
 #pragma unroll
         for (int c = 0; c < NCH; ++c) dsumc[c] += dd[c];
-        if (WIN && chunk_live) {
+        if (WINON && chunk_live) {
           // exact exit of token t2 = t + Tbar from the window: subtract W_i gC_{t2},
           // W_i = exp(A * sum_{j=i+1..t2} Delta_j); masked out when t2 >= T
           const float wm = j < nwin ? 1.f : 0.f;
@@ -1001,11 +1019,11 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         for (int ch = 0; ch < NCH; ++ch) {
           u64 sacc, dacc;
           u64 ach = 0ull;
-          if (SC && !PARK_ABAR) ach = ex2_2(mul2(d2[ch], A2[ch * 4]));   // scalar rate: one factor for the channel's states
+          if (SC) ach = ex2_2(mul2(d2[ch], A2[ch * 4]));   // scalar rate: one factor for the channel's states
 #pragma unroll
           for (int m = 0; m < 4; ++m) {
             const int u = ch * 4 + m;
-            const u64 a = PARK_ABAR ? aT[u] : (SC ? ach : ex2_2(mul2(d2[ch], A2[u])));
+            const u64 a = SC ? ach : ex2_2(mul2(d2[ch], A2[u]));
             const u64 hn = hT[u];                                  // h_i
             const u64 hb = fma2(ndx2[ch], Bp[m], hn);              // abar_i h_{i-1} = h_i - Delta_i x_i B_i
             vB[m] = ch == 0 ? mul2(mu[u], dx2[ch]) : fma2(mu[u], dx2[ch], vB[m]);   // dB partial (two channels)
@@ -1067,7 +1085,7 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         pD -= CH * 4; pX -= CH * ESZ; pB -= NBC; pR -= NBC;
       }
     }
-    if (WIN) {
+    if (WINON) {
 #pragma unroll
       for (int c = 0; c < NCH; ++c) sw[c] += (double)(dsumc[c] - sd2[c]);   // window sum at the previous chunk's last token
     }
@@ -1081,6 +1099,9 @@ adjoint_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
       if (j < nt) atomicAdd(dbc + ((int64_t)b * T + tc + j) * NBC + q, sum);
     }
   }
+  };
+  if (WIN && !seg_dead) walk_segment(std::integral_constant<bool, WIN>{});
+  else walk_segment(std::false_type{});
   if (failed) {
     if (w.tid == 0) {
       // copies already issued still target this CTA's shared memory: one more bounded wait for each before leaving
@@ -1163,10 +1184,10 @@ EncodeTiledFn get_encode() {
   }
   return fn;
 }
-int act_map(CUtensorMap* tm, const void* base, const Plan& pl, int elem_bytes, bool is_bf16) {
+int act_map(CUtensorMap* tm, const void* base, const Plan& pl, int batches, int elem_bytes, bool is_bf16) {
   EncodeTiledFn enc = get_encode();
   if (!enc) return 1;
-  cuuint64_t dims[2] = {(cuuint64_t)pl.P, (cuuint64_t)pl.B * (cuuint64_t)pl.T};
+  cuuint64_t dims[2] = {(cuuint64_t)pl.P, (cuuint64_t)batches * (cuuint64_t)pl.T};
   cuuint64_t strides[1] = {(cuuint64_t)pl.P * elem_bytes};
   cuuint32_t box[2] = {(cuuint32_t)CH, (cuuint32_t)CK};   // wider than P when P < CH: the rest is zero-filled
   cuuint32_t estr[2] = {1, 1};
@@ -1179,9 +1200,9 @@ struct Maps { CUtensorMap x, d, g; };
 int make_maps(const Plan& pl, const ScanPtrs& sp, Maps* m) {
   const bool bf = pl.io == AS_BF16;
   const int e = bf ? 2 : 4;
-  if (act_map(&m->x, sp.x, pl, e, bf)) return 1;
-  if (act_map(&m->d, sp.ws + pl.off_delta, pl, 4, false)) return 1;
-  if (act_map(&m->g, sp.dy ? sp.dy : sp.x, pl, e, bf)) return 1;
+  if (act_map(&m->x, sp.x, pl, pl.B, e, bf)) return 1;
+  if (act_map(&m->d, sp.ws + pl.off_delta, pl, pl.B, 4, false)) return 1;
+  if (act_map(&m->g, sp.dy ? sp.dy : sp.x, pl, sp.dy ? pl.Bg : pl.B, e, bf)) return 1;   // dy: one copy for all layers
   return 0;
 }
 

@@ -31,7 +31,7 @@ def test_exports_match_header(L):
 
 
 def test_version_and_strerror(L):
-    assert B.as_version() == 102
+    assert B.as_version() == 103
     assert B.strerror(0) == "ok"
     assert "tbar" in B.strerror(B.AS_ERR_TBAR)
     assert "unknown" in B.strerror(-999)
@@ -41,7 +41,7 @@ def test_struct_layout_matches_c():
     # int32, (pad), int64, 4 x int32  ->  32 bytes with natural alignment
     assert C.sizeof(B.as_shape_t) == 32
     assert B.as_shape_t.seqlen.offset == 8 and B.as_shape_t.d_model.offset == 16 and B.as_shape_t.a_structure.offset == 28
-    assert C.sizeof(B.as_params_t) == 40 and C.sizeof(B.as_grads_t) == 48
+    assert C.sizeof(B.as_params_t) == 48 and C.sizeof(B.as_grads_t) == 48
 
 
 def test_workspace_query_and_argument_errors(L):

@@ -43,6 +43,8 @@ def check_stack(io, K, T, P, tbar, mode, batch=2, config=4, every_layer=False):
     grads, G0 = st.adjoint_grad(g, mode, record=rec)
     torch.cuda.synchronize()
     assert B.as_check_status(st.ws) == B.AS_OK
+    if mode == "paper":
+        assert B.as_check_status(st.ws_last) == B.AS_OK
     ths = [theta_f64(t) for t in thetas]
     tol = TOL[io]
     for k, (yh, Gk) in rec.items():
@@ -74,7 +76,8 @@ def check_stack(io, K, T, P, tbar, mode, batch=2, config=4, every_layer=False):
     print(f"stack {io} K={K} T={T} P={P} tbar={tbar} {mode}: worst end-to-end relative L2 error {worst:.3e}")
 
 
-@pytest.mark.parametrize("io,K,T,P,tbar", [("f32", 3, 300, 40, 300), ("f32", 3, 300, 40, 50), ("bf16", 24, 1024, 128, 256)])
+@pytest.mark.parametrize("io,K,T,P,tbar", [("f32", 3, 300, 40, 300), ("f32", 3, 300, 40, 50), ("bf16", 24, 1024, 128, 256),
+                                           ("bf16", 4, 300, 64, 60)])
 @pytest.mark.parametrize("mode", ["chained", "paper"])
 def test_stack_gradients(io, K, T, P, tbar, mode):
     check_stack(io, K, T, P, tbar, mode)
@@ -86,25 +89,51 @@ def test_c4_width_stack_every_layer():
     check_stack("bf16", 24, 4096, 768, 1024, "chained", batch=1, every_layer=True)
 
 
-def test_paper_mode_on_two_streams_equals_one_stream():
-    """Prop. 3's layers are independent: spreading them over two streams (each with its own workspace) changes nothing
-    but the order of the fp32 atomic sums."""
-    K, T, P, tbar = 6, 1200, 128, 256
-    w = synth.custom_workload("stack2", 5, 2, T, P, layers=K, tbar=tbar, io="bf16")
+@pytest.mark.parametrize("io,K,T,P,tbar,with_dx", [("bf16", 5, 1024, 128, 256, True), ("bf16", 3, 300, 64, 50, False),
+                                                    ("f32", 3, 300, 40, 70, True)])
+def test_layers_call_equals_single_layer_calls(io, K, T, P, tbar, with_dx):
+    """as_adjoint_grad_layers (Prop. 3: all layers of the stack in one launch per phase) gives, layer by layer, what
+    as_adjoint_grad gives on that layer's parameters and input with the shared upstream gradient - for token counts
+    per layer that are (1024 x 2) and are not (300 x 2) a multiple of the 128-row contraction tile, and for fp32 I/O."""
+    w = synth.custom_workload("layers", 6, 2, T, P, layers=K, tbar=tbar, io=io)
     thetas = [synth.layer_params(w, k, DEV, slow_decay=True) for k in range(K)]
-    y0, g = synth.activations(w, DEV)
-    out = []
-    for ns in (1, 2):
-        st = Stack(thetas, w.batch, T, P, dtype=w.torch_dtype, device=DEV, tbar=tbar, paper_streams=ns)
-        st.forward(y0)
-        grads, _ = st.adjoint_grad(g, "paper")
-        torch.cuda.synchronize()
-        assert B.as_check_status(st.ws) == B.AS_OK
-        out.append(grads)
-    for a, b in zip(*out):
-        for k in O.PARAM_GRADS:
-            scale = float(a[k].abs().max())
-            assert float((a[k] - b[k]).abs().max()) <= 1e-2 * scale, k
+    _, g = synth.activations(w, DEV)
+    xs = torch.stack([synth.activations(synth.custom_workload("layers", 60 + k, 2, T, P, tbar=tbar, io=io), DEV)[0]
+                      for k in range(K)]).contiguous()
+    sh = B.shape_of(g)
+    stacked = {k: torch.stack([th[k] for th in thetas]).contiguous() for k in thetas[0]}
+    ws = B.alloc_workspace(B.as_workspace_bytes_layers(sh, K, tbar), DEV)
+    gl = B.alloc_grads_layers(sh, K, DEV, with_dx=with_dx)
+    B.as_adjoint_grad_layers(sh, K, stacked, xs, g, tbar, gl, ws)
+    assert B.as_check_status(ws) == B.AS_OK
+    torch.cuda.synchronize()
+    for k in range(K):
+        one = gpu_adjoint(w, thetas[k], xs[k].contiguous(), g, tbar, with_dx=with_dx)
+        ref = OP.batched_adjoint_grad(theta_f64(thetas[k]), synth.to_f64(xs[k]), synth.to_f64(g), tbar, tier="block",
+                                      channel_block=64)
+        for name in O.PARAM_GRADS + (("dx",) if with_dx else ()):
+            a, b_ = synth.to_f64(gl[name][k]), synth.to_f64(one[name])
+            assert np.abs(a - b_).max() <= 1e-5 * np.abs(b_).max() + 1e-30, (k, name)   # same kernels, other atomic order
+            assert_close(a, ref[name], TOL[io], f"layer {k} {name}")
+
+
+def test_packed_weights_handle_changes_nothing():
+    w = synth.custom_workload("wcat", 7, 2, 900, 96, tbar=200, io="bf16")
+    theta = synth.layer_params(w, 0, DEV)
+    x, dy = synth.activations(w, DEV)
+    sh = B.shape_of(x)
+    a = gpu_adjoint(w, theta, x, dy, w.tbar)
+    n0 = B.as_launch_count(reset=True)
+    gpu_adjoint(w, theta, x, dy, w.tbar)
+    with_pack = B.as_launch_count(reset=True)
+    th2 = dict(theta)
+    th2["Wcat"] = torch.empty(B.as_wcat_bytes(sh), dtype=torch.uint8, device=DEV)
+    B.as_pack_weights(sh, 1, theta, th2["Wcat"])
+    B.as_launch_count(reset=True)
+    b = gpu_adjoint(w, th2, x, dy, w.tbar)
+    assert B.as_launch_count(reset=True) == with_pack - 1      # the per-call packing kernel is gone
+    for k in O.PARAM_GRADS + ("dx",):
+        assert torch.equal(a[k], b[k]) or float((a[k].float() - b[k].float()).abs().max()) <= 1e-5 * float(a[k].float().abs().max()), k
 
 
 def oracle_batched(theta, x, dy, tbar, channel_block=64):
