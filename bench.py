@@ -159,7 +159,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C3")
-    ap.add_argument("--cpu-sample-tokens", type=int, default=16384)
+    ap.add_argument("--cpu-sample-tokens", type=int, default=32768)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--batch", type=int, default=None, help="override the workload's batch (profiling runs)")
@@ -333,10 +333,11 @@ def report(args, B, w, world, rank, tokens, ms, ms_e2e, h2d, d2h, launches, phas
         sm_mhz = (clocks or {}).get("sm_mhz") or 1965.0
         sms = B.as_sm_count()
         steps = tokens * P * N
+        ex2_steps = tokens * P if args.scalar_a else steps    # scalar structure: one decay factor per (token, channel)
         live = 1.0 if args.slow_decay else 0.0            # the window-exit factor is live under the slow-decay law only
-        ex2_method = steps * (METHOD_EX2_PER_STATE_STEP + live)
+        ex2_method = ex2_steps * (METHOD_EX2_PER_STATE_STEP + live)
         fma_method = steps * METHOD_FMA_PER_STATE_STEP
-        ex2_exec = steps * (sum(KERNEL_EX2_PER_STATE_STEP.values()) + live) + tokens * P      # + sigmoid per (token, channel)
+        ex2_exec = ex2_steps * (sum(KERNEL_EX2_PER_STATE_STEP.values()) + live) + tokens * P  # + sigmoid per (token, channel)
         mufu_peak = MUFU_PER_CLK_SM * sms * sm_mhz * 1e6
         fma_peak = FMA_PER_CLK_SM * sms * sm_mhz * 1e6
         sec = k_ms * 1e-3
