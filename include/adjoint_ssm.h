@@ -23,7 +23,7 @@
  *     (each call with its own `ws`), except for the phase-timing diagnostic (one thread, one stream) and the
  *     shared array of as_ssm_forward_static.  The library uses the CUDA runtime API, i.e. each device's primary context.
  *   - Size limits (AS_ERR_LIMIT): batch * seqlen + seqlen + 16 < 2^31 (token rows are 32-bit TMA coordinates) and
- *     seqlen <= 65535 * 2048 (time segments fill one grid dimension).
+ *     seqlen <= 65527 * 2048 (time segments fill one grid dimension).
  *   - Device-side waits: every wait on staged data (mbarrier waits on TMA / bulk copies and on tensor-core commits)
  *     is bounded and ends in AS_ERR_TIMEOUT.  The one wait that has no software bound is the hardware allocation of
  *     tensor memory (tcgen05.alloc) at the start of the contraction and adjoint kernels: it blocks until enough of

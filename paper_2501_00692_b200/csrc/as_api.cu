@@ -168,15 +168,18 @@ int check_grad_args(const as_shape_t* sh, const as_params_t* pr, const void* x, 
 
 int zero_outputs(const Plan& pl, uint32_t flags, const as_grads_t* out, char* ws, cudaStream_t st) {
   const size_t P = pl.P, K = pl.KL;
-  AS_TRY((int)cudaMemsetAsync(ws + pl.off_status, 0, 256, st));
-  AS_TRY((int)cudaMemsetAsync(ws + pl.off_dbc, 0, (size_t)pl.B * pl.T * NBC * 4, st));
+  ZeroList z{};
+  auto add = [&](void* p, size_t bytes) { z.ptr[z.n] = p; z.bytes[z.n] = (bytes + 15) / 16 * 16; ++z.n; };
+  add(ws + pl.off_status, 256);
+  add(ws + pl.off_dbc, (size_t)pl.B * pl.T * NBC * 4);
   if (!(flags & AS_ACCUMULATE)) {
-    AS_TRY((int)cudaMemsetAsync(out->dW_delta, 0, K * P * P * 4, st));
-    AS_TRY((int)cudaMemsetAsync(out->db_delta, 0, K * P * 4, st));
-    AS_TRY((int)cudaMemsetAsync(out->dW_B, 0, K * NS * P * 4, st));
-    AS_TRY((int)cudaMemsetAsync(out->dW_C, 0, K * NS * P * 4, st));
-    AS_TRY((int)cudaMemsetAsync(out->dA_log, 0, K * (pl.scalar ? P : P * NS) * 4, st));
+    add(out->dW_delta, K * P * P * 4);
+    add(out->db_delta, K * P * 4);
+    add(out->dW_B, K * NS * P * 4);
+    add(out->dW_C, K * NS * P * 4);
+    add(out->dA_log, K * (pl.scalar ? P : P * NS) * 4);
   }
+  AS_TRY(launch_zero_regions(z, st));
   return AS_OK;
 }
 

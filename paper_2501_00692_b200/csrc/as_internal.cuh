@@ -143,6 +143,10 @@ int launch_bptt(const Plan& pl, const ScanPtrs& sp, float* dA_log, float* db_del
 // device address of the library's built-in scratch array on the current device (as_noalloc.cu); AS_OK or an error code
 int static_scratch_address(void** out);
 
+// regions to clear in one launch (each 16-byte aligned, length a multiple of 16 bytes)
+struct ZeroList { void* ptr[8]; size_t bytes[8]; int n; };
+int launch_zero_regions(const ZeroList& z, cudaStream_t st);
+
 int launch_rmsnorm_fwd(const as_shape_t* sh, const void* y, void* yhat, float eps, cudaStream_t st);
 int launch_residual_add(const as_shape_t* sh, const void* a, const void* b, void* out, cudaStream_t st);
 int launch_rmsnorm_bwd_add(const as_shape_t* sh, const void* y, const void* dyhat, void* G, float eps,

@@ -86,4 +86,31 @@ int launch_residual_add(const as_shape_t* sh, const void* a, const void* b, void
   count_launch();
   return (int)cudaGetLastError();
 }
+
+// One launch clears every buffer a gradient call accumulates into (status block, the [dB|dC] accumulator and, unless
+// the caller accumulates, the five parameter gradients): seven separate memsets cost more in launch gaps than in
+// bytes.  All regions are 16-byte aligned and a multiple of 16 bytes long.
+namespace {
+__global__ void zero_regions_kernel(ZeroList z) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int r = 0; r < z.n; ++r) {
+    uint4* p = reinterpret_cast<uint4*>(z.ptr[r]);
+    const int64_t n16 = (int64_t)(z.bytes[r] / 16);
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += stride) p[i] = make_uint4(0u, 0u, 0u, 0u);
+  }
+}
+}  // namespace
+
+int launch_zero_regions(const ZeroList& z, cudaStream_t st) {
+  size_t total = 0;
+  for (int r = 0; r < z.n; ++r) total += z.bytes[r];
+  int64_t blocks = (int64_t)((total / 16 + 255) / 256);
+  const int64_t cap = (int64_t)sm_count() * 8;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  zero_regions_kernel<<<(unsigned)blocks, 256, 0, st>>>(z);
+  count_launch();
+  return (int)cudaGetLastError();
+}
+
 }  // namespace as

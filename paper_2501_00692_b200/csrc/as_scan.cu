@@ -79,7 +79,8 @@ int make_plan(const as_shape_t* sh, int64_t tbar, int layers, Plan* pl) {
   p.off_bptt_ckpt = take((size_t)p.B * ((p.T + 63) / 64) * p.P * NS * 4);
   p.total_grad = o;
   *pl = p;
-  return (p.S > 65535 || p.B > 65535) ? AS_ERR_LIMIT : AS_OK;   // segments fill gridDim.y, (layer, batch) gridDim.z
+  // segments (plus the NU blocks of the forward carry) fill gridDim.y, (layer, batch) gridDim.z
+  return (p.S > 65535 - NU || p.B > 65535) ? AS_ERR_LIMIT : AS_OK;
 }
 
 namespace {
@@ -482,10 +483,10 @@ __global__ void __launch_bounds__(NTHR, 4) ascend_kernel(const __grid_constant__
 // carries across segments.  Thread (b, tile, tid) owns the same 16 (channel, state) slots as in the scans.
 // ------------------------------------------------------------------------------------------------
 // hstart[s]: true state entering segment s (sequential in s).  The recurrence over segments is a chain of dependent
-// steps, so the kernel is latency-bound: one thread per state pair (blockIdx.z = the unit u of the scan kernels'
+// steps, so the kernel is latency-bound: one thread per state pair (u = the unit of the scan kernels'
 // thread), and the loads of a batch of 16 segments are issued together, one batch ahead of the one being applied.
-__global__ void __launch_bounds__(NTHR) fixup_h_kernel(Plan pl, const float* __restrict__ A_log, char* __restrict__ ws) {
-  const int tile = blockIdx.x, b = blockIdx.y, u = blockIdx.z;
+__device__ __forceinline__ void fixup_h_block(const Plan& pl, const float* __restrict__ A_log, char* __restrict__ ws,
+                                              int tile, int b, int u) {
   const Who w = who(tile, pl.P);
   A_log += (int64_t)(b / pl.Bg) * a_stride_dev(pl);
   u64 A2all[NU];
@@ -539,8 +540,8 @@ __global__ void __launch_bounds__(NTHR) fixup_h_kernel(Plan pl, const float* __r
 //   mu_loc[s+1] + D[s+1] (mu_loc[s+2] + ... + D[s+m] mu_part[s+m+1]),   D[s'] = exp(A * sum of Delta over s'),
 // i.e. m whole segments plus the first r tokens of the next one (all later segments in the full form).
 // swin[s]: sum of Delta over the Tbar tokens after e (fp64), for the window-exit factor.
-__global__ void __launch_bounds__(NTHR) fixup_mu_kernel(Plan pl, const float* __restrict__ A_log, char* __restrict__ ws) {
-  const int tile = blockIdx.x, b = blockIdx.z;
+__device__ __forceinline__ void fixup_mu_block(const Plan& pl, const float* __restrict__ A_log, char* __restrict__ ws,
+                                               int tile, int sy, int b) {
   const int P = pl.P, S = pl.S;
   const Who w = who(tile, P);
   A_log += (int64_t)(b / pl.Bg) * a_stride_dev(pl);
@@ -567,7 +568,7 @@ __global__ void __launch_bounds__(NTHR) fixup_mu_kernel(Plan pl, const float* __
     for (int u = 0; u < NU; ++u) val[u] = fma2(ex2_2(mul2(d2[u / 4], A2[u])), val[u], ml[u]);
   };
   if (pl.full) {
-    if (blockIdx.y != 0) return;
+    if (sy != 0) return;
     u64 val[NU];
 #pragma unroll
     for (int u = 0; u < NU; ++u) val[u] = 0ull;
@@ -576,7 +577,7 @@ __global__ void __launch_bounds__(NTHR) fixup_mu_kernel(Plan pl, const float* __
       step(s, val);
     }
   } else {
-    const int s = blockIdx.y;
+    const int s = sy;
     const int s1 = s + 1;
     u64 val[NU];
 #pragma unroll
@@ -602,6 +603,15 @@ __global__ void __launch_bounds__(NTHR) fixup_mu_kernel(Plan pl, const float* __
       for (int c = 0; c < NCH; ++c) dst[c] = swv[c] + (double)pv.v[c];
     }
   }
+}
+
+// Both carry computations in one launch (they are independent and each is latency-bound): blockIdx.y < ny_h runs the
+// forward carry for unit u = blockIdx.y, the rest the reverse carry for segment blockIdx.y - ny_h.
+__global__ void __launch_bounds__(NTHR) fixup_kernel(Plan pl, const float* __restrict__ A_log, char* __restrict__ ws,
+                                                     int ny_h) {
+  const int tile = blockIdx.x, b = blockIdx.z;
+  if ((int)blockIdx.y < ny_h) fixup_h_block(pl, A_log, ws, tile, b, (int)blockIdx.y);
+  else fixup_mu_block(pl, A_log, ws, tile, (int)blockIdx.y - ny_h, b);
 }
 
 // abar for the NU units of a thread from the per-channel exponent scale e2[ch] = {e, e}: exp2(e * A2[u]).  With a
@@ -1257,12 +1267,9 @@ int launch_prepass(const Plan& pl, const ScanPtrs& sp, bool with_mu, cudaStream_
 }
 
 int launch_fixup(const Plan& pl, const ScanPtrs& sp, bool with_mu, cudaStream_t st) {
-  fixup_h_kernel<<<dim3(pl.tiles, pl.B, NU), NTHR, 0, st>>>(pl, sp.A_log, sp.ws);
+  const int ny_mu = with_mu ? (pl.full ? 1 : pl.S) : 0;
+  fixup_kernel<<<dim3(pl.tiles, NU + ny_mu, pl.B), NTHR, 0, st>>>(pl, sp.A_log, sp.ws, NU);
   count_launch();
-  if (with_mu) {
-    fixup_mu_kernel<<<dim3(pl.tiles, pl.full ? 1 : pl.S, pl.B), NTHR, 0, st>>>(pl, sp.A_log, sp.ws);
-    count_launch();
-  }
   return (int)cudaGetLastError();
 }
 
