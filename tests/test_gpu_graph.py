@@ -1,4 +1,4 @@
-"""The gradient call is a pure stream of kernel launches and memsets: after one eager call (which sets the
+"""The gradient call is a pure stream of kernel launches: after one eager call (which sets the
 function attributes) it can be captured into a CUDA graph and replayed."""
 import pytest
 import torch
