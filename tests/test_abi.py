@@ -79,6 +79,25 @@ def test_workspace_query_and_argument_errors(L):
     assert L.as_adjoint_grad(C.byref(sh), C.byref(p), ok, ok, 0, 0, C.byref(g), ok, 1 << 40, None) == B.AS_ERR_TBAR
     assert L.as_full_bptt_grad(C.byref(sh), C.byref(p), ok, ok, 0, C.byref(g), ok, 1024, None) == B.AS_ERR_WORKSPACE
     assert L.as_rmsnorm_fwd(C.byref(sh), None, ok, 1e-6, None) == B.AS_ERR_NULL
+    # the layers call: same checks, plus the layer count and the limits on layers * batch
+    one = B.as_workspace_bytes(sh, 2048)[1]
+    many = B.as_workspace_bytes_layers(sh, 4, 2048)
+    assert B.as_workspace_bytes_layers(sh, 1, 2048) == one and 3 * one < many < 5 * one
+    assert L.as_adjoint_grad_layers(C.byref(sh), 0, C.byref(p), ok, ok, 4, 0, C.byref(g), ok, 1 << 40, None) == B.AS_ERR_SHAPE
+    assert L.as_adjoint_grad_layers(C.byref(sh), 3, C.byref(p), ok, ok, 4, 0, C.byref(g), ok, 1024, None) == B.AS_ERR_WORKSPACE
+    assert L.as_adjoint_grad_layers(C.byref(sh), 3, C.byref(p), None, ok, 4, 0, C.byref(g), ok, 1 << 40, None) == B.AS_ERR_NULL
+    for layers, shape in ((40000, B.make_shape(2, 64, 64)), (1 << 14, B.make_shape(1, 1 << 18, 8))):
+        with pytest.raises(B.AsError) as ei:
+            B.as_workspace_bytes_layers(shape, layers, 4)
+        assert ei.value.code == B.AS_ERR_LIMIT
+    # packed weights: size query and argument checks
+    assert B.as_wcat_bytes(sh, 3) == 3 * (768 + 32) * 768 * 2 and B.as_wcat_bytes(B.make_shape(0, 8, 64), 1) == 0
+    assert L.as_pack_weights(C.byref(sh), 1, C.byref(p), None, None) == B.AS_ERR_NULL
+    assert L.as_pack_weights(C.byref(sh), 0, C.byref(p), ok, None) == B.AS_ERR_SHAPE
+    f32 = B.make_shape(2, 64, 64)
+    assert L.as_pack_weights(C.byref(f32), 1, C.byref(p), ok, None) == B.AS_ERR_DTYPE
+    pw = B.as_params_t(ok, ok, ok, ok, ok, C.c_void_p(0x1008))
+    assert L.as_adjoint_grad(C.byref(sh), C.byref(pw), ok, ok, 4, 0, C.byref(g), ok, 1 << 40, None) == B.AS_ERR_ALIGN
 
 
 def test_missing_library_fails_loudly(monkeypatch):
