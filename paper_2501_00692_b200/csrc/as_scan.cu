@@ -37,9 +37,11 @@ int make_plan(const as_shape_t* sh, int64_t tbar, int layers, Plan* pl) {
   p.tiles = (p.P + CH - 1) / CH;
   p.bw = p.P < CH ? p.P : CH;
   const int64_t ctas = (int64_t)p.tiles * p.B;
-  // two full waves of the main kernel's resident CTAs (148 SMs x CTAs per SM), never more than that
+  // full waves of the main kernel's resident CTAs (SMs x CTAs per SM)
   const int64_t slots = (int64_t)sm_count() * 3;   // resident CTAs of the main kernel
-  int64_t s_target = (2 * slots) / ctas;
+  // three waves in the truncated form (shorter segments balance the tail better than they cost in carries); the
+  // full form's reverse carry is sequential over the segments, which favours fewer of them
+  int64_t s_target = ((p.full ? 2 : 3) * slots) / ctas;
   if (s_target < 1) s_target = 1;
   int64_t L = (p.T + s_target - 1) / s_target;
   L = (L + CK - 1) / CK * CK;
@@ -163,7 +165,7 @@ struct Stage {
 constexpr int NSTAGE = 3;        // ascending kernels
 constexpr int WRED_Q = 32 * 4 + 8;   // floats per quarter-block of the per-warp reduction scratch (512 B + 32 B skew)
 constexpr int MAIN_CTAS = 3;    // resident CTAs per SM the main kernel is compiled for (up to 168 registers per thread)
-constexpr int FW_UNROLL = 4;     // unroll factor of the main adjoint kernel's forward rebuild loop
+constexpr int FW_UNROLL = 8;     // unroll factor of the main adjoint kernel's forward rebuild loop (the whole chunk)
 constexpr int BW_UNROLL = 2;     // unroll factor of the main adjoint kernel's backward token loop
 constexpr int NSTAGE_MAIN = 2;   // main adjoint kernel: a chunk takes thousands of cycles, one chunk of lookahead suffices
 
