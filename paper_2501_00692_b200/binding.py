@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libadjoint_ssm.so")
 
 AS_F32, AS_BF16 = 0, 1
-AS_A_DIAGONAL, AS_A_SCALAR = 0, 1
+AS_A_DIAGONAL, AS_A_SCALAR, AS_A_SCALAR_MM = 0, 1, 2
 AS_ACCUMULATE = 1
 AS_OK = 0
 AS_ERR_NULL, AS_ERR_SHAPE, AS_ERR_DTYPE, AS_ERR_TBAR = -1, -2, -3, -4
@@ -117,9 +117,10 @@ def make_shape(batch, seqlen, d_model, d_state=16, io=AS_F32, a_structure=AS_A_D
     return as_shape_t(int(batch), int(seqlen), int(d_model), int(d_state), int(io), int(a_structure))
 
 
-def shape_of(x: torch.Tensor, d_state=16, a_scalar=False) -> as_shape_t:
+def shape_of(x: torch.Tensor, d_state=16, a_scalar=False, matmul_form=False) -> as_shape_t:
     io = {torch.float32: AS_F32, torch.bfloat16: AS_BF16}[x.dtype]
-    return make_shape(x.shape[0], x.shape[1], x.shape[2], d_state, io, AS_A_SCALAR if a_scalar else AS_A_DIAGONAL)
+    st = (AS_A_SCALAR_MM if matmul_form else AS_A_SCALAR) if a_scalar else AS_A_DIAGONAL
+    return make_shape(x.shape[0], x.shape[1], x.shape[2], d_state, io, st)
 
 
 def make_params(theta: dict) -> as_params_t:
@@ -133,7 +134,7 @@ def alloc_grads(shape: as_shape_t, device, with_dx=True) -> dict:
     f = dict(dtype=torch.float32, device=device)
     g = {"dW_delta": torch.empty(P, P, **f), "db_delta": torch.empty(P, **f), "dW_B": torch.empty(N, P, **f),
          "dW_C": torch.empty(N, P, **f),
-         "dA_log": torch.empty(P, **f) if shape.a_structure == AS_A_SCALAR else torch.empty(P, N, **f), "dx": None}
+         "dA_log": torch.empty(P, **f) if shape.a_structure != AS_A_DIAGONAL else torch.empty(P, N, **f), "dx": None}
     if with_dx:
         dt = torch.float32 if shape.io == AS_F32 else torch.bfloat16
         g["dx"] = torch.empty(shape.batch, shape.seqlen, P, dtype=dt, device=device)
@@ -217,7 +218,7 @@ def alloc_grads_layers(shape: as_shape_t, layers: int, device, with_dx=False) ->
     f = dict(dtype=torch.float32, device=device)
     g = {"dW_delta": torch.empty(K, P, P, **f), "db_delta": torch.empty(K, P, **f), "dW_B": torch.empty(K, N, P, **f),
          "dW_C": torch.empty(K, N, P, **f),
-         "dA_log": torch.empty(K, P, **f) if shape.a_structure == AS_A_SCALAR else torch.empty(K, P, N, **f), "dx": None}
+         "dA_log": torch.empty(K, P, **f) if shape.a_structure != AS_A_DIAGONAL else torch.empty(K, P, N, **f), "dx": None}
     if with_dx:
         dt = torch.float32 if shape.io == AS_F32 else torch.bfloat16
         g["dx"] = torch.empty(K, shape.batch, shape.seqlen, P, dtype=dt, device=device)

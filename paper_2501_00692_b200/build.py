@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libadjoint_ssm.so")
-SOURCES = ["as_api.cu", "as_gemm_simt.cu", "as_gemm_tc.cu", "as_scan.cu", "as_bptt.cu", "as_norm.cu", "as_noalloc.cu"]
+SOURCES = ["as_api.cu", "as_gemm_simt.cu", "as_gemm_tc.cu", "as_scan.cu", "as_scan_mm.cu", "as_bptt.cu", "as_norm.cu", "as_noalloc.cu"]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

@@ -27,7 +27,7 @@ int check_shape(const as_shape_t* sh) {
   if (!sh) return AS_ERR_NULL;
   if (sh->batch < 1 || sh->seqlen < 1 || sh->d_model < 1) return AS_ERR_SHAPE;
   if (sh->d_state != NS) return AS_ERR_SHAPE;
-  if (sh->a_structure != AS_A_DIAGONAL && sh->a_structure != AS_A_SCALAR) return AS_ERR_SHAPE;
+  if (sh->a_structure != AS_A_DIAGONAL && sh->a_structure != AS_A_SCALAR && sh->a_structure != AS_A_SCALAR_MM) return AS_ERR_SHAPE;
   if (sh->io != AS_F32 && sh->io != AS_BF16) return AS_ERR_DTYPE;
   if (sh->d_model % 8 != 0) return AS_ERR_ALIGN;
   if (sh->batch > 65535) return AS_ERR_SHAPE;
@@ -253,7 +253,8 @@ int as_ssm_forward(const as_shape_t* shape, const as_params_t* params, const voi
   ScanPtrs sp{x, nullptr, params->A_log, w};
   AS_TRY(launch_prepass(pl, sp, false, st));
   AS_TRY(launch_fixup(pl, sp, false, st));
-  AS_TRY(launch_forward_y(pl, sp, y, st));
+  if (forward_y_mm_applies(pl)) AS_TRY(launch_forward_y_mm(pl, sp, y, st));
+  else AS_TRY(launch_forward_y(pl, sp, y, st));
   return AS_OK;
 }
 

@@ -31,7 +31,7 @@ def test_exports_match_header(L):
 
 
 def test_version_and_strerror(L):
-    assert B.as_version() == 103
+    assert B.as_version() == 104
     assert B.strerror(0) == "ok"
     assert "tbar" in B.strerror(B.AS_ERR_TBAR)
     assert "unknown" in B.strerror(-999)
