@@ -26,7 +26,7 @@
  *     seqlen <= 65527 * 2048 (time segments fill one grid dimension).
  *   - Device-side waits: every wait on staged data (mbarrier waits on TMA / bulk copies and on tensor-core commits)
  *     is bounded and ends in AS_ERR_TIMEOUT.  The one wait that has no software bound is the hardware allocation of
- *     tensor memory (tcgen05.alloc) at the start of the contraction and adjoint kernels: it blocks until enough of
+ *     tensor memory (tcgen05.alloc) at the start of the contraction, adjoint and matmul-form forward kernels: it blocks until enough of
  *     the SM's 512 columns are free, which happens when CTAs that hold them finish; a kernel of this library frees
  *     its columns on every exit path and never waits for another CTA while holding them, so the allocation of a
  *     later CTA always completes.
