@@ -45,7 +45,7 @@ def _run(batch, T, P, slow=False, b_delta_range=None, config=31):
 
 
 @pytest.mark.parametrize("batch,T,P,slow", [(2, 2100, 256, False), (2, 2100, 256, True), (1, 64, 128, False),
-                                            (3, 65, 128, False), (2, 1000, 384, True)])
+                                            (3, 65, 128, False), (2, 10, 128, False), (2, 1000, 384, True)])
 def test_single_chunk_segments(batch, T, P, slow):
     y, ref = _run(batch, T, P, slow)
     assert_close(y, ref, TOL["bf16"], "y")
