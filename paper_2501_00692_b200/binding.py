@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libadjoint_ssm.so")
 
 AS_F32, AS_BF16 = 0, 1
-AS_A_DIAGONAL, AS_A_SCALAR, AS_A_SCALAR_MM = 0, 1, 2
+AS_A_DIAGONAL, AS_A_SCALAR = 0, 1
 AS_ACCUMULATE = 1
 AS_OK = 0
 AS_ERR_NULL, AS_ERR_SHAPE, AS_ERR_DTYPE, AS_ERR_TBAR = -1, -2, -3, -4
@@ -117,10 +117,9 @@ def make_shape(batch, seqlen, d_model, d_state=16, io=AS_F32, a_structure=AS_A_D
     return as_shape_t(int(batch), int(seqlen), int(d_model), int(d_state), int(io), int(a_structure))
 
 
-def shape_of(x: torch.Tensor, d_state=16, a_scalar=False, matmul_form=False) -> as_shape_t:
+def shape_of(x: torch.Tensor, d_state=16, a_scalar=False) -> as_shape_t:
     io = {torch.float32: AS_F32, torch.bfloat16: AS_BF16}[x.dtype]
-    st = (AS_A_SCALAR_MM if matmul_form else AS_A_SCALAR) if a_scalar else AS_A_DIAGONAL
-    return make_shape(x.shape[0], x.shape[1], x.shape[2], d_state, io, st)
+    return make_shape(x.shape[0], x.shape[1], x.shape[2], d_state, io, AS_A_SCALAR if a_scalar else AS_A_DIAGONAL)
 
 
 def make_params(theta: dict) -> as_params_t:

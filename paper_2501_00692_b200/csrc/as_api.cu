@@ -27,7 +27,7 @@ int check_shape(const as_shape_t* sh) {
   if (!sh) return AS_ERR_NULL;
   if (sh->batch < 1 || sh->seqlen < 1 || sh->d_model < 1) return AS_ERR_SHAPE;
   if (sh->d_state != NS) return AS_ERR_SHAPE;
-  if (sh->a_structure != AS_A_DIAGONAL && sh->a_structure != AS_A_SCALAR && sh->a_structure != AS_A_SCALAR_MM) return AS_ERR_SHAPE;
+  if (sh->a_structure != AS_A_DIAGONAL && sh->a_structure != AS_A_SCALAR) return AS_ERR_SHAPE;
   if (sh->io != AS_F32 && sh->io != AS_BF16) return AS_ERR_DTYPE;
   if (sh->d_model % 8 != 0) return AS_ERR_ALIGN;
   if (sh->batch > 65535) return AS_ERR_SHAPE;

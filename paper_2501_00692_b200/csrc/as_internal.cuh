@@ -92,7 +92,6 @@ struct Plan {
   int r;            // tbar % L   (tokens of the following partial segment)
   int io;           // as_dtype_t
   int scalar;       // 1: one decay rate per channel (A_log is [P]), 0: one per (channel, state)
-  int mm;           // 1: AS_A_SCALAR_MM - the forward's y pass runs in the matmul form where that applies
   int tiles;        // ceil(P / CH) channel tiles
   int bw;           // channels per staged row: min(CH, P)
   int tc;           // 1: bf16 tensor-core contractions (bf16 I/O and d_model % 32 == 0), 0: FP32-pipe GEMMs
@@ -129,7 +128,7 @@ struct ScanPtrs {
 int launch_prepass(const Plan& pl, const ScanPtrs& sp, bool with_mu, cudaStream_t st);
 int launch_fixup(const Plan& pl, const ScanPtrs& sp, bool with_mu, cudaStream_t st);
 int launch_forward_y(const Plan& pl, const ScanPtrs& sp, void* y, cudaStream_t st);
-// matmul form of the y pass (as_scan_mm.cu): AS_A_SCALAR_MM with bf16 I/O and d_model % 128 == 0
+// matmul form of the y pass (as_scan_mm.cu): scalar structure with bf16 I/O and d_model % 128 == 0
 bool forward_y_mm_applies(const Plan& pl);
 int launch_forward_y_mm(const Plan& pl, const ScanPtrs& sp, void* y, cudaStream_t st);
 int launch_adjoint_main(const Plan& pl, const ScanPtrs& sp, float* dA_log, float* db_delta, cudaStream_t st);

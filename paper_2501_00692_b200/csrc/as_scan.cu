@@ -29,8 +29,7 @@ int make_plan(const as_shape_t* sh, int64_t tbar, int layers, Plan* pl) {
   Plan p{};
   p.KL = layers < 1 ? 1 : layers; p.Bg = sh->batch;
   p.B = p.KL * p.Bg; p.P = sh->d_model; p.T = sh->seqlen; p.io = sh->io;
-  p.scalar = sh->a_structure != AS_A_DIAGONAL ? 1 : 0;
-  p.mm = sh->a_structure == AS_A_SCALAR_MM ? 1 : 0;
+  p.scalar = sh->a_structure == AS_A_SCALAR ? 1 : 0;
   p.tc = (sh->io == AS_BF16 && sh->d_model % 32 == 0) ? 1 : 0;
   p.du_ld = p.tc ? p.P + NBC : p.P;
   p.full = tbar >= p.T;

@@ -489,7 +489,7 @@ int chunk_map(CUtensorMap* tm, const void* base, const Plan& pl, int elem_bytes,
 
 }  // namespace
 
-bool forward_y_mm_applies(const Plan& pl) { return pl.mm && pl.scalar && pl.io == AS_BF16 && pl.P % MCH == 0; }
+bool forward_y_mm_applies(const Plan& pl) { return pl.scalar && pl.io == AS_BF16 && pl.P % MCH == 0; }
 
 int launch_forward_y_mm(const Plan& pl, const ScanPtrs& sp, void* y, cudaStream_t st) {
   CUtensorMap mx, md, my;

@@ -1,4 +1,4 @@
-"""Matmul form of the forward for the scalar structure (Table 1 "Scalar SSM"; AS_A_SCALAR_MM, bf16 I/O,
+"""Matmul form of the forward for the scalar structure (Table 1 "Scalar SSM"; what as_ssm_forward runs for bf16 I/O and
 d_model % 128 == 0) against the fp64 oracle's recurrence with the rates tied, through the C ABI (needs a B200).
 
 The cases cover chunks that are whole, ragged at the segment end and ragged at the sequence end, segments of several
@@ -31,7 +31,7 @@ def _run(batch, T, P, slow=False, b_delta_range=None, config=31):
     theta = dict(synth.layer_params(w, 0, DEV, slow_decay=slow, b_delta_range=b_delta_range))
     theta["A_log"] = theta["A_log"][:, 5].contiguous()            # [P]: the tied rate
     x, _ = synth.activations(w, DEV)
-    sh = B.shape_of(x, w.d_state, a_scalar=True, matmul_form=True)
+    sh = B.shape_of(x, w.d_state, a_scalar=True)
     fb, _ = B.as_workspace_bytes(sh, T)
     ws = B.alloc_workspace(fb, DEV)
     y = torch.full_like(x, float("nan"))
@@ -65,23 +65,7 @@ def test_large_steps_take_the_recurrence_per_channel(rng):
     assert_close(y, ref, TOL["bf16"], "y")
 
 
-def test_other_widths_and_the_gradient_entry_point_take_the_scan_kernels():
+def test_other_widths_take_the_scan_kernels():
     # d_model not a multiple of 128 keeps the scan kernels: same oracle, same bar
     y, ref = _run(2, 900, 96)
     assert_close(y, ref, TOL["bf16"], "y")
-    # as_adjoint_grad reads AS_A_SCALAR_MM as AS_A_SCALAR: the same kernels (sums by atomics: equal up to their order)
-    w = synth.custom_workload("scalar-mm", 33, 2, 700, 128, tbar=100, io="bf16")
-    theta = dict(synth.layer_params(w, 0, DEV))
-    theta["A_log"] = theta["A_log"][:, 5].contiguous()
-    x, dy = synth.activations(w, DEV)
-    outs = []
-    for mm in (False, True):
-        sh = B.shape_of(x, w.d_state, a_scalar=True, matmul_form=mm)
-        ws = B.alloc_workspace(B.as_workspace_bytes(sh, 100)[1], DEV)
-        g = B.alloc_grads(sh, DEV)
-        B.as_adjoint_grad(sh, theta, x, dy, 100, g, ws)
-        torch.cuda.synchronize()
-        assert B.as_check_status(ws) == 0
-        outs.append(g)
-    for k in O.PARAM_GRADS + ("dx",):
-        assert_close(synth.to_f64(outs[1][k]), synth.to_f64(outs[0][k]), 1e-3, k)
