@@ -50,7 +50,7 @@ typedef enum { AS_F32 = 0, AS_BF16 = 1 } as_dtype_t;
 /* Structure of A (Table 1 of Section 4.5): AS_A_DIAGONAL, one decay rate per (channel, state), A_log [P,N];
  * AS_A_SCALAR, one decay rate per channel shared by its N states ("Scalar SSM": A^t is a multiple of the identity on
  * each channel), A_log [P] and dA_log [P] (the sum over n of the diagonal layer's dA_log[p,n]).  With AS_A_SCALAR,
- * io == AS_BF16 and d_model % 128 == 0, as_ssm_forward computes y in the matmul form this structure admits (chunks of
+ * io == AS_BF16 and d_model % 128 == 0, as_ssm_forward runs its scans in the matmul form this structure admits (chunks of
  * 64 tokens as tensor-core products of tril(C B^T) with the decay-scaled inputs, state carried in tensor memory);
  * every other shape and every other entry point uses the scan kernels. */
 typedef enum { AS_A_DIAGONAL = 0, AS_A_SCALAR = 1 } as_structure_t;

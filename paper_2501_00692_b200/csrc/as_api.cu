@@ -251,9 +251,11 @@ int as_ssm_forward(const as_shape_t* shape, const as_params_t* params, const voi
   e = projections(pl, params, wcat, x, w, st);
   if (e) return e;
   ScanPtrs sp{x, nullptr, params->A_log, w};
-  AS_TRY(launch_prepass(pl, sp, false, st));
+  const bool mm = forward_y_mm_applies(pl);
+  if (mm) AS_TRY(launch_forward_state_mm(pl, sp, st));
+  else AS_TRY(launch_prepass(pl, sp, false, st));
   AS_TRY(launch_fixup(pl, sp, false, st));
-  if (forward_y_mm_applies(pl)) AS_TRY(launch_forward_y_mm(pl, sp, y, st));
+  if (mm) AS_TRY(launch_forward_y_mm(pl, sp, y, st));
   else AS_TRY(launch_forward_y(pl, sp, y, st));
   return AS_OK;
 }

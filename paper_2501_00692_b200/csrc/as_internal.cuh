@@ -131,6 +131,7 @@ int launch_forward_y(const Plan& pl, const ScanPtrs& sp, void* y, cudaStream_t s
 // matmul form of the y pass (as_scan_mm.cu): scalar structure with bf16 I/O and d_model % 128 == 0
 bool forward_y_mm_applies(const Plan& pl);
 int launch_forward_y_mm(const Plan& pl, const ScanPtrs& sp, void* y, cudaStream_t st);
+int launch_forward_state_mm(const Plan& pl, const ScanPtrs& sp, cudaStream_t st);   // the segment pass in the same form
 int launch_adjoint_main(const Plan& pl, const ScanPtrs& sp, float* dA_log, float* db_delta, cudaStream_t st);
 int launch_wait_selftest(int* status, unsigned limit, cudaStream_t st);
 int launch_finish_dx(const Plan& pl, const float* dxacc, const void* dxdir, void* dx, cudaStream_t st);

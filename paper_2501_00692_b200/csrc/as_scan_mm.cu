@@ -151,15 +151,18 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 // operand descriptor for the rows from `row` on (a multiple of 8) and the K columns from 16*kstep on
 __device__ __forceinline__ uint64_t desc_at(uint32_t tile, int row, int kstep) { return make_desc(tile + row * 128 + kstep * 32); }
 
+// YPASS: the y pass from the true segment-start state.  !YPASS: the segment pass of the forward (local scan from a zero
+// state: only V and the state products), which writes the segment's end state and Delta sum for the carry kernel.
+template <bool YPASS>
 __global__ void __launch_bounds__(MT, 2)
-scalar_y_mm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmD,
+scalar_mm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmD,
                    const __grid_constant__ CUtensorMap tmY, Plan pl, const float* __restrict__ A_log,
                    char* __restrict__ ws, __nv_bfloat16* __restrict__ y) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_ld, bar_g, bar_y;
   __shared__ uint32_t tmem_base_s;
   __shared__ float xch[4][MCH];   // per channel: Delta sums (to the reference, of the whole half) of half 0 and of half 1
-  __shared__ int slow_s[MCH];     // per channel: 1 if either half left the factorised form in this chunk
+  __shared__ int slow_s[2][MCH];  // per channel and half: 1 if the half left the factorised form in this chunk
   uint8_t* sm = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // stays a shared-space pointer
 
   const int tile = blockIdx.x, s = blockIdx.y, b = blockIdx.z;
@@ -195,7 +198,7 @@ scalar_y_mm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
   float S[NS];
 #pragma unroll
   for (int n = 0; n < NS; ++n) S[n] = 0.f;
-  if (hf == 0) {
+  if (YPASS && hf == 0) {
     const float* hst = reinterpret_cast<const float*>(ws + pl.off_hstart) +
                        (((int64_t)b * pl.S + s) * pl.tiles + tile) * TILE_FLOATS;
 #pragma unroll
@@ -205,6 +208,8 @@ scalar_y_mm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
   float xprev = 1.f, fprev = 1.f;   // thread (p, 0): the factors that take S0 and S1 of the previous chunk to its end
   const uint32_t sm_b = smem_u32(sm);
   bool failed = false;
+  bool prefetched = false;      // the coming chunk's tiles are already on their way (CTA-uniform)
+  float seg_sum = 0.f;          // !YPASS, thread (p, 0): Delta sum of the segment so far
 
   // [B | C] rows of the coming chunk, 8 values per thread: token tid & 63, part tid >> 6 = (B 0..7, B 8..15, C 0..7, C 8..15)
   const int bt = tid & 63, bpart = tid >> 6;
@@ -223,18 +228,20 @@ scalar_y_mm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     const int64_t tc = t0 + (int64_t)c * TCK;
     const int nt = (int)min((int64_t)TCK, t1 - tc);
     const int64_t row0 = (int64_t)b * T + tc;
-    if (tid == 0) {
-      bulk_wait_read_all();   // the previous chunk's y tile has left the x buffer
+    if (tid == 0 && !prefetched) {
+      if (YPASS) bulk_wait_read_all();   // the previous chunk's y tile has left the x buffer
       mbar_expect_tx(&bar_ld, TCK * MCH * 2 + TCK * MCH * 4);
       tma_2d(sm + SM_X, &tmX, tile * MCH, row0, &bar_ld);
       tma_2d(sm + SM_D, &tmD, tile * MCH, row0, &bar_ld);
     }
+    prefetched = false;
     // ---- [B | C] rows -> bf16 operand tiles (rows past the segment end are zeros) ----
     {
       const float v[8] = {bcr[0].x, bcr[0].y, bcr[0].z, bcr[0].w, bcr[1].x, bcr[1].y, bcr[1].z, bcr[1].w};
       uint8_t* dst = sm + (bpart >= 2 ? SM_CT : SM_BT);
-      *reinterpret_cast<uint4*>(dst + sw128(bt, bpart & 1)) =
-          make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+      if (YPASS)
+        *reinterpret_cast<uint4*>(dst + sw128(bt, bpart & 1)) =
+            make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
       if (bpart < 2) {
 #pragma unroll
         for (int n = 0; n < 8; ++n)
@@ -244,7 +251,7 @@ scalar_y_mm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     }
     bool ok = mbar_wait(&bar_ld, c & 1);
     if (__syncthreads_or(ok ? 0 : 1)) { failed = true; break; }
-    if (tid == 0) {   // G = C B^T into lanes 0..63 of columns 0..63 (issued as 128 x 64: rows 64.. of the A tile are never looked at)
+    if (YPASS && tid == 0) {   // G = C B^T into lanes 0..63 of columns 0..63 (issued as 128 x 64: rows 64.. of the A tile are never looked at)
       tc_fence_after();
       umma_bf16(tm + TM_D, make_desc(sm_b + SM_CT), make_desc(sm_b + SM_BT), idesc_n(64), 0u);
       umma_commit(&bar_g);
@@ -291,7 +298,7 @@ scalar_y_mm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     const bool slow_half = fmaxf(cs_r, cs_t - cs_r) * -a2 > EXP_LIMIT;
     xch[2 * hf][pc] = cs_r;
     xch[2 * hf + 1][pc] = cs_t;
-    if (hf == 0) slow_s[pc] = 0;
+    slow_s[hf][pc] = slow_half ? 1 : 0;
     // ---- thread (p, 0): state at the chunk start, brought to the reference point of half 0, handed to the GEMMs ----
     if (hf == 0) {   // warps 0..3, warp-uniform
       if (c > 0) {   // the TMEM loads are warp-collective: every lane takes them, a lane whose state is in registers keeps it
@@ -310,18 +317,30 @@ scalar_y_mm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
 #pragma unroll
       for (int n = 0; n < NS; ++n) { sp[n] = S[n] * f; r[n] = __float_as_uint(sp[n]); }
       tmem_st16(tm_lane + TM_S0, r);
-      *reinterpret_cast<uint4*>(sm + SM_SP + sw128(pc, 0)) =
-          make_uint4(pack_bf16(sp[0], sp[1]), pack_bf16(sp[2], sp[3]), pack_bf16(sp[4], sp[5]), pack_bf16(sp[6], sp[7]));
-      *reinterpret_cast<uint4*>(sm + SM_SP + sw128(pc, 1)) =
-          make_uint4(pack_bf16(sp[8], sp[9]), pack_bf16(sp[10], sp[11]), pack_bf16(sp[12], sp[13]), pack_bf16(sp[14], sp[15]));
+      if (YPASS) {
+        *reinterpret_cast<uint4*>(sm + SM_SP + sw128(pc, 0)) =
+            make_uint4(pack_bf16(sp[0], sp[1]), pack_bf16(sp[2], sp[3]), pack_bf16(sp[4], sp[5]), pack_bf16(sp[6], sp[7]));
+        *reinterpret_cast<uint4*>(sm + SM_SP + sw128(pc, 1)) =
+            make_uint4(pack_bf16(sp[8], sp[9]), pack_bf16(sp[10], sp[11]), pack_bf16(sp[12], sp[13]), pack_bf16(sp[14], sp[15]));
+      }
     }
     fence_async_smem();
     tc_fence_before();
-    __syncthreads();
-    if (slow_half) slow_s[pc] = 1;   // benign race: both halves may write the same 1
+    const int any_slow = __syncthreads_or(slow_half ? 1 : 0);
+    const bool slow = (slow_s[0][pc] | slow_s[1][pc]) != 0;
+    if (!YPASS && !any_slow && c + 1 < nchunk) {
+      // the segment pass is done with the x and Delta tiles once V is written (no channel needs them for a recurrence):
+      // the next chunk's tiles travel while this chunk's products run
+      if (tid == 0) {
+        mbar_expect_tx(&bar_ld, TCK * MCH * 2 + TCK * MCH * 4);
+        tma_2d(sm + SM_X, &tmX, tile * MCH, row0 + TCK, &bar_ld);
+        tma_2d(sm + SM_D, &tmD, tile * MCH, row0 + TCK, &bar_ld);
+      }
+      prefetched = true;
+    }
 
     // ---- G (TMEM lanes 0..63 = tokens t) -> lower triangle -> bf16 operand rows ----
-    if (warp < 2) {
+    if (YPASS && warp < 2) {
       ok = mbar_wait(&bar_g, c & 1);
       if (ok) {
         tc_fence_after();
@@ -346,12 +365,14 @@ scalar_y_mm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         fence_async_smem();
       }
     }
-    tc_fence_before();
-    if (__syncthreads_or(ok ? 0 : 1)) { failed = true; break; }
-    const bool slow = slow_s[pc] != 0;
+    if (YPASS) {
+      tc_fence_before();
+      if (__syncthreads_or(ok ? 0 : 1)) { failed = true; break; }
+    }
     if (tid == 0) {
       tc_fence_after();
       const uint32_t V = sm_b + SM_V, GM = sm_b + SM_GM, CT = sm_b + SM_CT, SP = sm_b + SM_SP, BTT = sm_b + SM_BTT;
+      if (YPASS) {
       // half 0:  V0 G00^T + S' C0^T
       umma_bf16(tm + TM_D, desc_at(V, 0, 0), desc_at(GM, 0, 0), idesc_n(32), 0u);
       umma_bf16(tm + TM_D, desc_at(V, 0, 1), desc_at(GM, 0, 1), idesc_n(32), 1u);
@@ -363,6 +384,7 @@ scalar_y_mm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       umma_bf16(tm + TM_D + 64, desc_at(V, 0, 0), desc_at(GM, 32, 0), idesc_n(32), 0u);
       umma_bf16(tm + TM_D + 64, desc_at(V, 0, 1), desc_at(GM, 32, 1), idesc_n(32), 1u);
       umma_bf16(tm + TM_D + 64, desc_at(SP, 0, 0), desc_at(CT, 32, 0), idesc_n(32), 1u);
+      }
       // state:  S0 = S' + V0^T B0,  S1 = V1^T B1
       umma_bf16(tm + TM_S0, desc_at(V, 0, 0), desc_at(BTT, 0, 0), idesc_n(16), 1u);
       umma_bf16(tm + TM_S0, desc_at(V, 0, 1), desc_at(BTT, 0, 1), idesc_n(16), 1u);
@@ -372,12 +394,22 @@ scalar_y_mm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     }
     // while the products run: the next chunk's [B | C] rows, and the factors this thread needs below
     if (c + 1 < nchunk) fetch_bc(row0 + TCK, (int)min((int64_t)TCK, t1 - tc - TCK));
+    if (!YPASS && hf == 0 && slow) {
+      // this channel left the factorised form in this chunk: its state by the plain recurrence (B as the bf16 operand holds it)
+      for (int t = 0; t < nt; ++t) {
+        const float d = dcol[t * MCH];
+        const float ab = ex2_approx(a2 * d), dx = d * __bfloat162float(xcol[t * MCH]);
+#pragma unroll
+        for (int n = 0; n < NS; ++n)
+          S[n] = fmaf(ab, S[n], dx * __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + SM_BTT + sw128(n, t >> 3) + (t & 7) * 2)));
+      }
+    }
     const float c0r = xch[0][pc], c0t = xch[1][pc], c1r = xch[2][pc], c1t = xch[3][pc];
     const float xoff = (c0t - c0r) + c1r;   // Delta sum between the two reference points
     ok = mbar_wait(&bar_y, c & 1);
     // ---- epilogue: thread (p, h) finishes its 32 tokens of channel p; y goes to the staging tile [t][p] ----
     __nv_bfloat16* ycol = reinterpret_cast<__nv_bfloat16*>(sm + SM_X) + (HCK * hf) * MCH + pc;   // the x tile is consumed
-    if (ok) {
+    if (YPASS && ok) {
       tc_fence_after();
       uint32_t r[32], r2[32];
       tmem_ld32(tm_lane + TM_D + 32 * hf, r);
@@ -427,15 +459,17 @@ scalar_y_mm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
           ycol[t * MCH] = __float2bfloat16_rn(acc);
         }
       }
-      if (hf == 0) {   // bookkeeping of thread (p, 0) for the next chunk's state
-        s_in_regs = slow;
-        xprev = ex2_approx(a2 * (xoff + (c1t - c1r)));   // exp(a (cs_end - cs_r0)): takes S0 to the chunk end
-        fprev = ex2_approx(a2 * (c1t - c1r));            // exp(a (cs_end - cs_r1)): takes S1 there
-      }
+    }
+    if (hf == 0) {   // bookkeeping of thread (p, 0) for the next chunk's state
+      s_in_regs = slow;
+      xprev = ex2_approx(a2 * (xoff + (c1t - c1r)));   // exp(a (cs_end - cs_r0)): takes S0 to the chunk end
+      fprev = ex2_approx(a2 * (c1t - c1r));            // exp(a (cs_end - cs_r1)): takes S1 there
+      seg_sum += c0t + c1t;
     }
     fence_async_smem();
     tc_fence_before();
     if (__syncthreads_or(ok ? 0 : 1)) { failed = true; break; }
+    if (!YPASS) continue;
     if (nt == TCK) {
       if (tid == 0) { tma_store_2d(&tmY, sm + SM_X, tile * MCH, row0); bulk_commit(); }
     } else {
@@ -443,6 +477,23 @@ scalar_y_mm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       for (int t = 0; t < nth; ++t) y[(row0 + HCK * hf + t) * P + pch] = ycol[t * MCH];
       __syncthreads();   // before the next chunk's x lands in this buffer
     }
+  }
+  if (!YPASS && !failed && hf == 0) {
+    // end state of the local scan and the segment's Delta sum, in the layout the carry kernel reads
+    if (nchunk > 0) {   // warp-collective loads: every lane takes them
+      uint32_t r0[16], r1[16];
+      tc_fence_after();
+      tmem_ld16(tm_lane + TM_S0, r0);
+      tmem_ld16(tm_lane + TM_S1, r1);
+      if (!s_in_regs) {
+#pragma unroll
+        for (int n = 0; n < NS; ++n) S[n] = fmaf(xprev, __uint_as_float(r0[n]), fprev * __uint_as_float(r1[n]));
+      }
+    }
+    float* hend = reinterpret_cast<float*>(ws + pl.off_hend) + (((int64_t)b * pl.S + s) * pl.tiles + tile) * TILE_FLOATS;
+#pragma unroll
+    for (int n = 0; n < NS; ++n) hend[tile_block_offset(pc, n)] = S[n];
+    reinterpret_cast<float*>(ws + pl.off_segd)[((int64_t)b * pl.S + s) * P + pch] = seg_sum;
   }
   if (tid == 0) {
     bulk_wait_all();
@@ -496,10 +547,22 @@ int launch_forward_y_mm(const Plan& pl, const ScanPtrs& sp, void* y, cudaStream_
   if (chunk_map(&mx, sp.x, pl, 2, true, MCH, false)) return 1;
   if (chunk_map(&md, sp.ws + pl.off_delta, pl, 4, false, MCH, false)) return 1;
   if (chunk_map(&my, y, pl, 2, true, MCH, false)) return 1;
-  auto kern = scalar_y_mm_kernel;
+  auto kern = scalar_mm_kernel<true>;
   static bool done[AS_MAX_DEVICES] = {};
   if (ensure_dynamic_smem(kern, SMEM_DYN, done)) return 1;
   kern<<<dim3(pl.P / MCH, pl.S, pl.B), MT, SMEM_DYN, st>>>(mx, md, my, pl, sp.A_log, sp.ws, (__nv_bfloat16*)y);
+  count_launch();
+  return (int)cudaGetLastError();
+}
+
+int launch_forward_state_mm(const Plan& pl, const ScanPtrs& sp, cudaStream_t st) {
+  CUtensorMap mx, md;
+  if (chunk_map(&mx, sp.x, pl, 2, true, MCH, false)) return 1;
+  if (chunk_map(&md, sp.ws + pl.off_delta, pl, 4, false, MCH, false)) return 1;
+  auto kern = scalar_mm_kernel<false>;
+  static bool done[AS_MAX_DEVICES] = {};
+  if (ensure_dynamic_smem(kern, SMEM_DYN, done)) return 1;
+  kern<<<dim3(pl.P / MCH, pl.S, pl.B), MT, SMEM_DYN, st>>>(mx, md, mx, pl, sp.A_log, sp.ws, nullptr);
   count_launch();
   return (int)cudaGetLastError();
 }
