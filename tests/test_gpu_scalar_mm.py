@@ -58,6 +58,12 @@ def test_segments_of_several_chunks_with_ragged_tails():
     assert_close(y, ref, TOL["bf16"], "y")
 
 
+def test_c5_width_segments_of_six_chunks():
+    # 16 channel tiles of the widest workload; segments of 368 tokens = five whole chunks and one of 48
+    y, ref = _run(1, 20000, 2048, config=5)
+    assert_close(y, ref, TOL["bf16"], "y")
+
+
 @pytest.mark.parametrize("rng", [(1.0, 3.0), (-3.0, 1.0), (-1.0, 1.0)])
 def test_large_steps_take_the_recurrence_per_channel(rng):
     # Delta of order one: |a| times half a chunk's Delta sum passes the exponent bound for most or some channels
