@@ -75,3 +75,30 @@ def test_other_widths_take_the_scan_kernels():
     # d_model not a multiple of 128 keeps the scan kernels: same oracle, same bar
     y, ref = _run(2, 900, 96)
     assert_close(y, ref, TOL["bf16"], "y")
+
+
+def test_c3_full_size_sampled_channels():
+    """Workload C3 at full size with the rates tied (segments of 888 tokens = 13 whole chunks and one of 56, the launch
+    configuration the forward benchmark times): y[:, :, p] against the oracle's scan for 32 sampled channels p."""
+    from oracle_parallel import _fwd_block, map_bounded, _scan_gb
+    w = synth.WORKLOADS["C3"]
+    theta = dict(synth.layer_params(w, 0, DEV))
+    theta["A_log"] = theta["A_log"][:, 5].contiguous()
+    x, _ = synth.activations(w, DEV)
+    sh = B.shape_of(x, w.d_state, a_scalar=True)
+    ws = B.alloc_workspace(B.as_workspace_bytes(sh, w.seqlen)[0], DEV)
+    y = torch.full_like(x, float("nan"))
+    B.as_ssm_forward(sh, theta, x, y, ws)
+    torch.cuda.synchronize()
+    assert B.as_check_status(ws) == 0
+    assert torch.isfinite(y.float()).all()
+    rng = np.random.default_rng(3)
+    sel = np.unique(np.concatenate([[0, 127, 128, w.d_model - 1], rng.choice(w.d_model, 28, replace=False)]))[:32]
+    th = O.untie_scalar_A(theta_f64(theta), w.d_state)
+    th_sel = dict(th, W_delta=th["W_delta"][sel], b_delta=th["b_delta"][sel], A_log=th["A_log"][sel])
+    for b in range(w.batch):
+        _, delta, Bm, Cm, A = O.nets(th_sel, synth.to_f64(x[b]))
+        xsel = synth.to_f64(x[b][:, sel])
+        jobs = [(delta[:, c:c + 8], xsel[:, c:c + 8], Bm, Cm, A[c:c + 8]) for c in range(0, len(sel), 8)]
+        yref = np.concatenate(map_bounded(_fwd_block, jobs, _scan_gb(w.seqlen, 8, w.d_state) / 2), axis=1)
+        assert_close(synth.to_f64(y[b][:, sel]), yref, TOL["bf16"], f"y[{b}, :, sel]")
